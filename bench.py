@@ -1,0 +1,399 @@
+#!/usr/bin/env python
+"""Benchmark of the KV-rebuild hot path on B200: prefix prefill into a paged cache, suffix pack,
+unpack/assemble and the resumed decode step, through the C ABI.
+
+  python bench.py --gpus N --steps K --warmup W            (N > 1: launched by torch.distributed.run)
+  python bench.py --impl reference ...                     (the CPU oracle on a bounded sample)
+
+One "step" is one pass of the whole path for one request of the workload.  Every rank runs an independent
+replica (the path does not shard: no data-path collective), so scaling is weak and `value` is the sum of
+the ranks' prefix tokens divided by the slowest rank's time.  Prints ONE JSON line on rank 0.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import synth  # noqa: E402
+
+METRIC = "prefix_kv_rebuild_tokens_per_s"
+UNIT = "tokens/s"
+# profiling recipe fallbacks when MEASURED_PEAKS.json is absent
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+FALLBACK_BF16_TFLOPS_SUSTAINED = 1400.0
+
+WORKLOADS = {
+    # name: (shape, prefix tokens, suffix tokens, pool blocks)
+    "32b-4k": ("32b", 4096, 512, 4096),
+    "8b-1k": ("8b", 1024, 256, 1024),
+    "tiny": ("tiny", 128, 32, 64),
+}
+
+# DRAM bytes (read + write) of one gate/up GEMM launch at the 32b-4k workload, from the ncu capture
+# summarised under profiles/ (None until a capture exists for the current kernel).
+NCU_TRAFFIC_BYTES = {"32b-4k": None}
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": FALLBACK_BF16_TFLOPS,
+            "bf16_tflops_sustained": FALLBACK_BF16_TFLOPS_SUSTAINED, "source": "fallback"}
+
+
+def prefill_flops(shape, n_tokens, with_logits=False):
+    """Executed flops of a K/V-only prefill: the last layer stops after its QKV projection."""
+    d, qd, kvd, f, L = shape.hidden, shape.q_dim, shape.kv_dim, shape.ffn, shape.n_layers
+    qkv = 2.0 * n_tokens * d * (qd + 2 * kvd)
+    rest = 2.0 * n_tokens * (qd * d + 3 * d * f)
+    attn = 2.0 * shape.n_q_heads * shape.head_dim * n_tokens * (n_tokens + 1)   # causal: N(N+1)/2 pairs, QK and PV
+    full_layers = L if with_logits else L - 1
+    return L * qkv + full_layers * (rest + attn)
+
+
+# ------------------------------------------------------------------------------------------ reference arm
+def oracle_sample(shape, n_tokens, seed=0):
+    """Bounded sample of the workload for the CPU oracle: ONE decoder layer over the first n_tokens prefix tokens."""
+    from oracle import kv_oracle as O
+    w = synth.layer_weights(shape, seed, 0)
+    x = (np.random.default_rng(seed).standard_normal((n_tokens, shape.hidden)) * shape.init_std)
+    pos = np.arange(n_tokens)
+
+    def run():
+        t0 = time.perf_counter()
+        O.layer_forward(shape, w, x, pos)
+        return time.perf_counter() - t0
+    return run
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 0) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else os.cpu_count()
+    except Exception:
+        return os.cpu_count()
+
+
+def cpu_baseline(shape, prefix, sample_tokens, repeats=1):
+    run = oracle_sample(shape, sample_tokens)
+    secs = min(run() for _ in range(repeats))
+    value = sample_tokens / (secs * shape.n_layers)
+    return {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+            "sample": f"one decoder layer (1 of {shape.n_layers}) of the fp64 numpy oracle over the first "
+                      f"{sample_tokens} of {prefix} prefix tokens, {secs:.2f} s; tokens/s extrapolated to "
+                      f"{shape.n_layers} layers",
+            "seconds": secs}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    shape_name, prefix, suffix, _ = WORKLOADS[args.workload]
+    shape = synth.SHAPES[shape_name]
+    sample_tokens = min(prefix, args.ref_tokens)
+    run = oracle_sample(shape, sample_tokens)
+    for _ in range(args.ref_warmup):
+        run()
+    times = [run() for _ in range(args.steps)]
+    secs = sum(times) / len(times)
+    value = sample_tokens / (secs * shape.n_layers)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.ref_warmup, "ms_per_step": secs * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "prefix_tokens": prefix, "suffix_tokens": suffix,
+                   "step": f"one decoder layer of {shape.n_layers} over {sample_tokens} prefix tokens (bounded sample)"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                         "sample": f"1 of {shape.n_layers} layers, {sample_tokens} of {prefix} prefix tokens, "
+                                   f"extrapolated to full depth"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# ------------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu_index)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, power, reasons = [], [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        with open(self.path) as f:
+            for line in f:
+                p = [x.strip() for x in line.split(",")]
+                if len(p) < 9:
+                    continue
+                try:
+                    sm.append(float(p[1])); mx.append(float(p[2])); power.append(float(p[3]))
+                except ValueError:
+                    continue
+                for name, val in zip(names, p[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        os.unlink(self.path)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_max": float(max(power))}
+
+
+# ------------------------------------------------------------------------------------------ our arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2608_16477_b200 as kv
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    kv.load()
+
+    shape_name, prefix, suffix, pool_blocks = WORKLOADS[args.workload]
+    shape = synth.SHAPES[shape_name]
+    if args.layers:
+        shape = shape.with_layers(args.layers)
+    bs = shape.block_size
+    n = prefix + suffix
+    seed = 1000 + rank
+    gen = torch.Generator(device="cuda").manual_seed(seed)
+
+    def mat(rows, cols):
+        return torch.empty(rows, cols, dtype=torch.bfloat16, device="cuda").normal_(0.0, shape.init_std, generator=gen)
+
+    def layer(l):
+        ones = torch.ones(shape.hidden, dtype=torch.bfloat16, device="cuda")
+        return {"attn_norm": ones, "ffn_norm": ones.clone(), "w_qkv": mat(shape.qkv_dim, shape.hidden),
+                "w_o": mat(shape.hidden, shape.q_dim), "w_gate_up": mat(2 * shape.ffn, shape.hidden),
+                "w_down": mat(shape.hidden, shape.ffn)}
+    head = {"embed": mat(shape.vocab, shape.hidden), "lm_head": mat(shape.vocab, shape.hidden),
+            "final_norm": torch.ones(shape.hidden, dtype=torch.bfloat16, device="cuda")}
+    model = kv.Model(shape, head, layer)
+
+    ids = synth.token_ids(shape, seed, n + 1)
+    src = kv.PagedCache(shape, pool_blocks)
+    tgt = kv.PagedCache(shape, pool_blocks, fill=0)
+    kv.kv_fill_pattern(src.data, src.data.numel() * 2, seed=seed)        # source pool holds arbitrary KV bytes
+    perm_src = synth.block_permutation(seed + 1, pool_blocks)
+    perm_tgt = synth.block_permutation(seed + 2, pool_blocks)
+    nb_prefix, nb_total = prefix // bs, -(-n // bs)
+    nb_suffix = nb_total - nb_prefix
+    tgt_prefix = perm_tgt[:nb_prefix].copy()
+    dst_ids = perm_tgt[nb_prefix:nb_total].copy()
+    extra = [int(perm_tgt[nb_total])] if n % bs == 0 else []
+    logical = np.arange(nb_prefix, nb_total, dtype=np.int32)
+    src_suffix = perm_src[nb_prefix:nb_total].copy()
+    wire_elems = nb_suffix * shape.n_layers * 2 * (src.page_bytes // 2)
+    wire = torch.empty(wire_elems, dtype=torch.int16, device="cuda")
+    wire2 = torch.empty_like(wire)
+    wire_host = torch.empty(wire_elems, dtype=torch.int16, pin_memory=True)
+    logits = torch.empty(shape.vocab, dtype=torch.float32, device="cuda")
+    logits_host = torch.empty(shape.vocab, dtype=torch.float32, pin_memory=True)
+    ws_p = model.workspace(kv.KV_OP_PREFILL, prefix)
+    ws_d = model.workspace(kv.KV_OP_DECODE, n + 1)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        kv.kv_prefill_prefix(model, tgt, ids[:prefix], tgt_prefix, workspace=ws_p)
+        kv.kv_pack_blocks(src, src_suffix, wire)
+        merged = kv.kv_unpack_assemble(tgt, wire, logical, dst_ids, tgt_prefix, n, epoch=1, expected_epoch=1)
+        kv.kv_decode_step(model, tgt, int(ids[n]), n, list(merged) + extra, logits, workspace=ws_d)
+
+    def step_e2e():
+        # host buffers: token ids and tables are host arrays; the wire crosses the host (the link between
+        # source and target) and the logits are read back
+        kv.kv_prefill_prefix(model, tgt, ids[:prefix], tgt_prefix, workspace=ws_p)
+        kv.kv_pack_blocks(src, src_suffix, wire)
+        wire_host.copy_(wire, non_blocking=True)
+        wire2.copy_(wire_host, non_blocking=True)
+        merged = kv.kv_unpack_assemble(tgt, wire2, logical, dst_ids, tgt_prefix, n, epoch=1, expected_epoch=1)
+        kv.kv_decode_step(model, tgt, int(ids[n]), n, list(merged) + extra, logits, workspace=ws_d)
+        logits_host.copy_(logits, non_blocking=True)
+        stream.synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            fn()
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    kv.kv_check_device_status(ws_p)
+    kv.kv_check_device_status(ws_d)
+    torch.cuda.synchronize()
+    kv.kv_profile_read()
+
+    sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else
+                           int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank]) if
+                           os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank].isdigit() else local_rank)
+    sampler.start()
+    kv.kv_profile_enable(True)
+    launches0 = kv.kv_launch_count()
+    total_ms = timed(step, args.steps)
+    launches = kv.kv_launch_count() - launches0
+    kv.kv_profile_enable(False)
+    prof = kv.kv_profile_read()
+    clocks = sampler.stop()
+    kv.kv_check_device_status(ws_p)
+    kv.kv_check_device_status(ws_d)
+
+    step_e2e()
+    e2e_ms = timed(step_e2e, args.steps)
+
+    # standalone pack / unpack bandwidth, rotating over disjoint block sets so every launch reads cold pages
+    n_sets = max(1, min(8, (pool_blocks - nb_total - 1) // max(nb_suffix, 1)))
+    sets_src = [perm_src[nb_total + 1 + i * nb_suffix: nb_total + 1 + (i + 1) * nb_suffix].copy() for i in range(n_sets)]
+    sets_dst = [perm_tgt[nb_total + 1 + i * nb_suffix: nb_total + 1 + (i + 1) * nb_suffix].copy() for i in range(n_sets)]
+    wires = [torch.empty(wire_elems, dtype=torch.int16, device="cuda") for _ in range(n_sets)]
+    payload = wire_elems * 2
+
+    def pack_all():
+        for i in range(n_sets):
+            kv.kv_pack_blocks(src, sets_src[i], wires[i])
+
+    def unpack_all():
+        for i in range(n_sets):
+            kv.kv_unpack_assemble(tgt, wires[i], logical, sets_dst[i], tgt_prefix, n, epoch=1, expected_epoch=1)
+    pack_all(); unpack_all()
+    reps = 5
+    pack_ms = timed(pack_all, reps) / (reps * n_sets)
+    unpack_ms = timed(unpack_all, reps) / (reps * n_sets)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    pk = peaks()
+    ms_per_step = total_ms / args.steps
+    value = world * prefix / (ms_per_step * 1e-3)
+    per_step = {k: (ms / args.steps, cnt // args.steps) for k, (ms, cnt) in prof.items()}
+    prefill_kinds = ("embed", "rmsnorm", "gemm_qkv", "rope_store", "attention", "gemm_o", "gemm_gate_up", "gemm_down")
+    prefill_ms = sum(per_step[k][0] for k in prefill_kinds)
+    decode_ms = sum(per_step[k][0] for k in ("decode_gemv", "decode_attention", "decode_other", "lm_head"))
+    gu_ms, gu_launches = prof["gemm_gate_up"]
+    gu_flops = 2.0 * prefix * shape.hidden * 2 * shape.ffn
+    achieved = gu_flops / (gu_ms / max(gu_launches, 1) * 1e-3) / 1e12 if gu_ms > 0 else 0.0
+    flops = prefill_flops(shape, prefix)
+    roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel<SWIGLU> (gate/up projection)", "achieved": achieved,
+                "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": achieved / pk["bf16_tflops_sustained"],
+                "frac_of_burst_peak": achieved / pk["bf16_tflops"], "peak_source": pk["source"] + " (sustained)",
+                "flops_per_launch": gu_flops, "launches_timed": gu_launches,
+                "traffic": NCU_TRAFFIC_BYTES.get(args.workload) if not args.layers else None}
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "shape": shape.name, "layers": shape.n_layers,
+                   "prefix_tokens": prefix, "suffix_tokens": suffix, "block_size": bs, "pool_blocks": pool_blocks,
+                   "block_ids": "seeded permutation (fragmented)", "parallelism": f"replicas x{world}",
+                   "l2": "inputs larger than L2: each step streams every weight (>> 126 MB) between "
+                         "consecutive launches of any kernel; standalone pack/unpack rotate over disjoint block sets"},
+        "clocks": clocks,
+        "e2e": {"value": world * prefix / (e2e_ms / args.steps * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": int(payload + 4 * (prefix + nb_prefix + nb_total + 1 + nb_suffix * 2)),
+                "d2h_bytes_per_step": int(payload + 4 * shape.vocab), "ms_per_step": e2e_ms / args.steps},
+        "gpu_launches": int(launches),
+        "roofline": roofline,
+        "prefill": {"ms_per_prefix": prefill_ms, "tokens_per_s": prefix / (prefill_ms * 1e-3),
+                    "tflops": flops / (prefill_ms * 1e-3) / 1e12,
+                    "frac_of_bf16_burst_peak": flops / (prefill_ms * 1e-3) / 1e12 / pk["bf16_tflops"],
+                    "frac_of_bf16_sustained_peak": flops / (prefill_ms * 1e-3) / 1e12 / pk["bf16_tflops_sustained"]},
+        "pack": {"gbs": 2 * payload / (pack_ms * 1e-3) / 1e9, "frac_of_hbm": 2 * payload / (pack_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
+                 "us": pack_ms * 1e3, "payload_bytes": payload},
+        "unpack": {"gbs": 2 * payload / (unpack_ms * 1e-3) / 1e9,
+                   "frac_of_hbm": 2 * payload / (unpack_ms * 1e-3) / 1e9 / pk["hbm_gbs"], "us": unpack_ms * 1e3},
+        "decode_step_ms": decode_ms,
+        "t0_analog_ms": per_step["unpack"][0] + decode_ms,
+        "breakdown_ms_per_step": {k: round(v[0], 4) for k, v in per_step.items()},
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(synth.SHAPES[shape_name], prefix, min(prefix, args.ref_tokens))
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="32b-4k", choices=sorted(WORKLOADS))
+    ap.add_argument("--layers", type=int, default=0, help="debug: reduced depth (invalid as a bench number)")
+    ap.add_argument("--ref-tokens", type=int, default=2048, help="prefix tokens in the oracle's bounded sample")
+    ap.add_argument("--ref-warmup", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -145,9 +145,21 @@ def _mm(x: np.ndarray, w: np.ndarray, mm_dtype) -> np.ndarray:
     return (np.asarray(x, dtype=mm_dtype) @ np.asarray(w, dtype=mm_dtype).T).astype(np.float64)
 
 
+def _act(x: np.ndarray, act_bf16: bool) -> np.ndarray:
+    """Optional bfloat16 storage point: the value as it exists after being stored in bf16."""
+    return from_bf16_bits(to_bf16_bits(x)).astype(np.float64) if act_bf16 else x
+
+
 def layer_forward(shape, w: dict, x: np.ndarray, positions: np.ndarray,
-                  k_past=None, v_past=None, mm_dtype=np.float64, skip_after_kv: bool = False):
+                  k_past=None, v_past=None, mm_dtype=np.float64, skip_after_kv: bool = False,
+                  act_bf16: bool = False):
     """One decoder layer on rows x [T, D] at absolute `positions`.
+
+    act_bf16 = False is the exact definition.  With act_bf16 every tensor that a 16-bit pipeline
+    stores between contractions (normed activations, post-RoPE Q/K and V, attention output,
+    SwiGLU output) is rounded to bfloat16 at that point while all arithmetic stays fp64: the
+    same function evaluated at bf16 storage precision, which separates rounding that the
+    2-byte cache/activation format makes unavoidable from arithmetic error.
 
     k_past/v_past: [P, Hkv, d] K/V of positions 0..P-1 already in the cache (None: P = 0);
     positions must equal P .. P+T-1.  Returns (x_out, k_new, v_new); k_new is post-RoPE.
@@ -156,13 +168,13 @@ def layer_forward(shape, w: dict, x: np.ndarray, positions: np.ndarray,
     """
     t = x.shape[0]
     hq, hkv, d = shape.n_q_heads, shape.n_kv_heads, shape.head_dim
-    h = rmsnorm(x, w["attn_norm"], shape.rms_eps)
+    h = _act(rmsnorm(x, w["attn_norm"], shape.rms_eps), act_bf16)
     qkv = _mm(h, w["w_qkv"], mm_dtype)
     q = qkv[:, : hq * d].reshape(t, hq, d)
     k = qkv[:, hq * d: (hq + hkv) * d].reshape(t, hkv, d)
-    v = qkv[:, (hq + hkv) * d:].reshape(t, hkv, d)
-    q = rope(q, positions, shape.rope_base)
-    k = rope(k, positions, shape.rope_base)
+    v = _act(qkv[:, (hq + hkv) * d:].reshape(t, hkv, d), act_bf16)
+    q = _act(rope(q, positions, shape.rope_base), act_bf16)
+    k = _act(rope(k, positions, shape.rope_base), act_bf16)
     if skip_after_kv:
         return None, k, v
     if k_past is not None and len(k_past):
@@ -170,17 +182,17 @@ def layer_forward(shape, w: dict, x: np.ndarray, positions: np.ndarray,
         v_all = np.concatenate([np.asarray(v_past, dtype=np.float64), v], axis=0)
     else:
         k_all, v_all = k, v
-    o = attention(q, k_all, v_all, q_pos0=int(positions[0]))
+    o = _act(attention(q, k_all, v_all, q_pos0=int(positions[0])), act_bf16)
     x = x + _mm(o.reshape(t, hq * d), w["w_o"], mm_dtype)
-    h2 = rmsnorm(x, w["ffn_norm"], shape.rms_eps)
+    h2 = _act(rmsnorm(x, w["ffn_norm"], shape.rms_eps), act_bf16)
     ab = _mm(h2, w["w_gate_up"], mm_dtype)
-    m = silu(ab[:, : shape.ffn]) * ab[:, shape.ffn:]
+    m = _act(silu(ab[:, : shape.ffn]) * ab[:, shape.ffn:], act_bf16)
     x = x + _mm(m, w["w_down"], mm_dtype)
     return x, k, v
 
 
 def forward_full(shape, head: dict, layers, token_ids, mm_dtype=np.float64,
-                 want_logits: bool = True, all_logits: bool = False):
+                 want_logits: bool = True, all_logits: bool = False, act_bf16: bool = False):
     """Full-sequence forward over token_ids[0..T).
 
     `layers` is a callable l -> weight dict (so large models are generated layer by layer).
@@ -195,7 +207,8 @@ def forward_full(shape, head: dict, layers, token_ids, mm_dtype=np.float64,
     ks, vs = [], []
     for l in range(shape.n_layers):
         last = (l == shape.n_layers - 1) and not want_logits
-        x, k, v = layer_forward(shape, layers(l), x, pos, mm_dtype=mm_dtype, skip_after_kv=last)
+        x, k, v = layer_forward(shape, layers(l), x, pos, mm_dtype=mm_dtype, skip_after_kv=last,
+                                act_bf16=act_bf16)
         ks.append(k)
         vs.append(v)
     logits = None

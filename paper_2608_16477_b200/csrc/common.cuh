@@ -1,0 +1,103 @@
+// Shared host/device helpers of the kvrebuild library (internal).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/kvrebuild.h"
+
+namespace kvr {
+
+typedef __nv_bfloat16 bf16;
+
+// Geometry of a paged cache as the kernels see it (byte strides).
+struct CacheView {
+  char *base;
+  long long layer_stride, kv_stride, block_stride;
+  int block_size, n_kv_heads, head_dim;
+  __host__ __device__ long long page_bytes() const { return (long long)block_size * n_kv_heads * head_dim * 2; }
+  __device__ __forceinline__ char *page(int layer, int kv, int block) const {
+    return base + layer * layer_stride + kv * kv_stride + block * block_stride;
+  }
+};
+
+inline CacheView make_view(const kv_cache_desc *c) {
+  CacheView v;
+  v.base = (char *)c->base_dev;
+  v.layer_stride = c->layer_stride;
+  v.kv_stride = c->kv_stride;
+  v.block_stride = c->block_stride;
+  v.block_size = c->block_size;
+  v.n_kv_heads = c->n_kv_heads;
+  v.head_dim = c->head_dim;
+  return v;
+}
+
+// Layout of the device status word block at the start of every prefill/decode workspace.
+struct DeviceStatus {
+  int error;      // 0, or the code of the first bounded wait that ran out
+  int where;      // kernel-specific tag of that wait
+  int detail[6];
+};
+
+void set_cuda_error(cudaError_t e, const char *what);
+
+// Number of kernels launched by this library so far (host counter, bumped by every launcher).
+extern long long g_launches;
+#define KV_COUNT_LAUNCH() (++::kvr::g_launches)
+
+// Kernel classes reported by the optional event profiler (kv_profile_*).
+enum ProfKind {
+  PROF_EMBED = 0, PROF_RMSNORM, PROF_GEMM_QKV, PROF_ROPE_STORE, PROF_ATTENTION, PROF_GEMM_O, PROF_GEMM_GATE_UP,
+  PROF_GEMM_DOWN, PROF_LM_HEAD, PROF_PACK, PROF_UNPACK, PROF_DECODE_GEMV, PROF_DECODE_ATTENTION, PROF_DECODE_OTHER,
+  PROF_KINDS
+};
+#define KV_CUDA(call)                                  \
+  do {                                                 \
+    cudaError_t e__ = (call);                          \
+    if (e__ != cudaSuccess) {                          \
+      ::kvr::set_cuda_error(e__, #call);               \
+      return KV_ERR_CUDA;                              \
+    }                                                  \
+  } while (0)
+
+// ---- launchers implemented in the .cu files (all enqueue on `st` and return a status) ----
+enum GemmMode { GEMM_STORE_BF16 = 0, GEMM_RESID_F32 = 1, GEMM_SWIGLU = 2, GEMM_QKV_ROPE = 3 };
+
+// Extra arguments of the fused QKV epilogue: RoPE on the accumulators, K/V stored into the paged cache.
+struct QkvRopeArgs {
+  const float2 *rope;       // [n_tokens, head_dim/2] (cos, sin) of positions pos0 .. pos0+n_tokens-1
+  const int *block_table;   // device
+  CacheView cache;
+  int pos0, head_dim, n_q_heads, n_kv_heads, layer;
+};
+
+int gemm_tc(const bf16 *a, int lda, const bf16 *w, int m, int n, int k, int mode, bf16 *out,
+            float *resid, int *status_dev, cudaStream_t st, const QkvRopeArgs *qkv_args = nullptr);
+int gemm_simt(const bf16 *a, int lda, const bf16 *w, int m, int n, int k, int mode, bf16 *out,
+              float *resid, cudaStream_t st);
+
+int embed_rows(const bf16 *embed, const int *ids_dev, int n_tokens, int hidden, float *x, cudaStream_t st);
+int rmsnorm_rows(const float *x, const bf16 *gain, int rows, int dim, float eps, bf16 *out, cudaStream_t st);
+int rope_table(float2 *table, int pos0, int n_tokens, int head_dim, float base, cudaStream_t st);
+int attention_prefill(const bf16 *qkv, int n_tokens, int pos0, int n_q_heads, int n_kv_heads,
+                      int head_dim, CacheView cache, int layer, const int *block_table_dev, bf16 *out,
+                      int *status_dev, cudaStream_t st);
+
+// decode-step kernels (one token, fp32 activations)
+int embed_one(const bf16 *embed, int token, int hidden, float *x, cudaStream_t st);
+int rmsnorm_vec(const float *x, const bf16 *gain, int dim, float eps, float *out, cudaStream_t st);
+// y[n] (+)= sum_k W[n,k] x[k]; mode 0 store, 1 add into y, 2 swiglu over (gate | up) rows
+int gemv(const bf16 *w, const float *x, int n, int k, int mode, float *y, cudaStream_t st);
+int rope_store_kv_one(float *qkv, int pos, int n_q_heads, int n_kv_heads, int head_dim, float base,
+                      CacheView cache, int layer, const int *block_table_dev, cudaStream_t st);
+long long paged_attention_scratch_bytes(int n_q_heads, int head_dim, int n_ctx);
+int paged_attention(const float *q, int n_q_heads, CacheView cache, int layer, const int *block_table_dev,
+                    int n_ctx, void *scratch, float *out, cudaStream_t st);
+
+int copy_pages(CacheView cache, int n_layers, const int *ids_host, int n_blocks, char *wire,
+               int wire_layout, int total_blocks_in_wire, int first_block_in_wire, bool to_wire,
+               cudaStream_t st);
+int fill_pattern(void *dst, long long bytes, unsigned long long seed, long long offset, cudaStream_t st);
+
+}  // namespace kvr

@@ -1,0 +1,100 @@
+// Bandwidth-bound steps of the prefill path: embedding gather, RMSNorm, RoPE table.
+#include "common.cuh"
+
+namespace kvr {
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// block-wide sum for blockDim.x <= 1024 (multiple of 32); every thread gets the result
+__device__ __forceinline__ float block_sum(float v, float *red) {
+  v = warp_sum(v);
+  const int w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  if ((threadIdx.x & 31) == 0) red[w] = v;
+  __syncthreads();
+  float t = (threadIdx.x & 31) < nw ? red[threadIdx.x & 31] : 0.f;
+  t = warp_sum(t);
+  __syncthreads();
+  return t;
+}
+
+// x[t, :] = float(E[ids[t], :])
+__global__ void embed_rows_kernel(const bf16 *__restrict__ embed, const int *__restrict__ ids, int hidden,
+                                  float *__restrict__ x) {
+  const int t = blockIdx.x;
+  const uint4 *src = reinterpret_cast<const uint4 *>(embed + (long long)ids[t] * hidden);
+  float4 *dst = reinterpret_cast<float4 *>(x + (long long)t * hidden);
+  for (int v = threadIdx.x; v < hidden / 8; v += blockDim.x) {
+    uint4 raw = src[v];
+    const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+    float2 a = __bfloat1622float2(h[0]), b = __bfloat1622float2(h[1]);
+    float2 c = __bfloat1622float2(h[2]), d = __bfloat1622float2(h[3]);
+    dst[2 * v] = make_float4(a.x, a.y, b.x, b.y);
+    dst[2 * v + 1] = make_float4(c.x, c.y, d.x, d.y);
+  }
+}
+
+int embed_rows(const bf16 *embed, const int *ids_dev, int n_tokens, int hidden, float *x, cudaStream_t st) {
+  embed_rows_kernel<<<n_tokens, 128, 0, st>>>(embed, ids_dev, hidden, x);
+  KV_COUNT_LAUNCH();
+  KV_CUDA(cudaGetLastError());
+  return KV_OK;
+}
+
+// out[r, :] = bf16( x[r, :] * rsqrt(mean(x[r, :]^2) + eps) * gain ), statistics in fp32.
+// One CTA per row; the row is read twice (second read served by L1/L2).
+__global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const float *__restrict__ x,
+                                                           const bf16 *__restrict__ gain, int dim, float eps,
+                                                           bf16 *__restrict__ out) {
+  __shared__ float red[32];
+  const float4 *row = reinterpret_cast<const float4 *>(x + (long long)blockIdx.x * dim);
+  float ss = 0.f;
+  for (int v = threadIdx.x; v < dim / 4; v += blockDim.x) {
+    float4 a = row[v];
+    ss += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
+  }
+  ss = block_sum(ss, red);
+  const float inv = rsqrtf(ss / (float)dim + eps);
+  __nv_bfloat162 *o = reinterpret_cast<__nv_bfloat162 *>(out + (long long)blockIdx.x * dim);
+  const __nv_bfloat162 *g = reinterpret_cast<const __nv_bfloat162 *>(gain);
+  for (int v = threadIdx.x; v < dim / 4; v += blockDim.x) {
+    float4 a = row[v];
+    float2 g0 = __bfloat1622float2(g[2 * v]), g1 = __bfloat1622float2(g[2 * v + 1]);
+    o[2 * v] = __floats2bfloat162_rn(a.x * inv * g0.x, a.y * inv * g0.y);
+    o[2 * v + 1] = __floats2bfloat162_rn(a.z * inv * g1.x, a.w * inv * g1.y);
+  }
+}
+
+int rmsnorm_rows(const float *x, const bf16 *gain, int rows, int dim, float eps, bf16 *out, cudaStream_t st) {
+  if (rows <= 0) return KV_OK;
+  rmsnorm_rows_kernel<<<rows, 256, 0, st>>>(x, gain, dim, eps, out);
+  KV_COUNT_LAUNCH();
+  KV_CUDA(cudaGetLastError());
+  return KV_OK;
+}
+
+// table[t, j] = (cos, sin)(pos * base^(-2j/d)), angle formed in fp64 so that positions in the
+// tens of thousands keep full fp32 accuracy after the final rounding.
+__global__ void rope_table_kernel(float2 *table, int pos0, int n_tokens, int half, float base) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= n_tokens * half) return;
+  const int t = idx / half, j = idx - t * half;
+  const double theta = pow((double)base, -(double)j / (double)half);
+  double s, c;
+  sincos((double)(pos0 + t) * theta, &s, &c);
+  table[idx] = make_float2((float)c, (float)s);
+}
+
+int rope_table(float2 *table, int pos0, int n_tokens, int head_dim, float base, cudaStream_t st) {
+  const int n = n_tokens * (head_dim / 2);
+  if (n <= 0) return KV_OK;
+  rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(table, pos0, n_tokens, head_dim / 2, base);
+  KV_COUNT_LAUNCH();
+  KV_CUDA(cudaGetLastError());
+  return KV_OK;
+}
+
+}  // namespace kvr

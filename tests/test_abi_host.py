@@ -1,0 +1,147 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every declared symbol,
+and rejects bad arguments before anything is enqueued (fake device addresses are never dereferenced)."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+import synth
+from oracle import kv_oracle as O
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def kv():
+    import paper_2608_16477_b200 as kv
+    kv.load()
+    return kv
+
+
+def test_exports_match_header(kv):
+    text = open(os.path.join(ROOT, "include", "kvrebuild.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    declared = set(re.findall(r"\b(kv_[a-z0-9_]+)\s*\(", text))
+    assert declared == set(kv.EXPORTS)
+    lib = kv.load()
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_status_codes_agree_with_oracle(kv):
+    pairs = {"OK": 0, "ERR_ARG": -1, "ERR_SHAPE": -2, "ERR_BLOCK_RANGE": -3, "ERR_BLOCK_ALIAS": -4, "ERR_GAP": -5,
+             "ERR_OVERLAP": -6, "ERR_SPLIT_UNALIGNED": -7, "ERR_TABLE_SHORT": -8, "ERR_WIRE_SIZE": -9,
+             "ERR_WORKSPACE": -10, "ERR_STALE_EPOCH": -11, "ERR_TOKEN_RANGE": -12}
+    text = open(os.path.join(ROOT, "include", "kvrebuild.h")).read()
+    for name, val in pairs.items():
+        assert getattr(O, name) == val
+        assert re.search(rf"KV_{name}\s*=\s*{val}\b", text), name
+        assert kv.status_string(val) != "unknown status"
+
+
+def test_eq1_through_abi(kv):
+    assert kv.kv_bytes_per_token(64, 8, 128, 2) == 262144 == O.kv_bytes_per_token(64, 8, 128, 2)
+
+
+class _FakeCache:
+    """Cache descriptor over a fake device address; only host-side validation may look at it."""
+
+    def __init__(self, kv, shape, num_blocks, base=0x7000000000):
+        from paper_2608_16477_b200.binding import CacheDesc
+        page = synth.kv_page_bytes(shape)
+        self.block_size = shape.block_size
+        self.desc = CacheDesc(base, 2 * num_blocks * page, num_blocks * page, page, num_blocks, shape.block_size,
+                              shape.n_layers, shape.n_kv_heads, shape.head_dim, 2)
+
+
+class _FakeBuf:
+    def __init__(self, nbytes, ptr=0x7100000000):
+        self._n, self._p = nbytes, ptr
+
+    def data_ptr(self): return self._p
+    def numel(self): return self._n
+    def element_size(self): return 1
+
+
+def _status(fn, *a, **k):
+    from paper_2608_16477_b200 import KVError
+    try:
+        fn(*a, **k)
+    except KVError as e:
+        return e.status
+    return 0
+
+
+def test_assemble_rejections_match_oracle(kv):
+    s = synth.SHAPES["tiny"]
+    cache = _FakeCache(kv, s, 12)
+    page = synth.kv_page_bytes(s)
+    wire = _FakeBuf(2 * s.n_layers * 2 * page)
+    base = dict(logical=[2, 3], dst=[5, 6], prefix=[0, 1], n=64, epoch=3, expected=3)
+    cases = [dict(epoch=2), dict(dst=[5, 12]), dict(dst=[5, -1]), dict(dst=[5, 5]), dict(dst=[5, 1]),
+             dict(logical=[2, 2]), dict(logical=[1, 3]), dict(logical=[2, 4]), dict(n=65)]
+    for c in cases:
+        a = {**base, **c}
+        want = O.check_assemble(12, s.block_size, a["logical"], a["dst"], a["prefix"], a["n"], a["epoch"], a["expected"])
+        got = _status(kv.kv_unpack_assemble, cache, wire, a["logical"], a["dst"], a["prefix"], a["n"],
+                      epoch=a["epoch"], expected_epoch=a["expected"], stream=0)
+        assert want != 0 and got == want, (c, got, want)
+    short = _FakeBuf(2 * s.n_layers * 2 * page - 16)
+    assert _status(kv.kv_unpack_assemble, cache, short, [2, 3], [5, 6], [0, 1], 64, stream=0) == O.ERR_WIRE_SIZE
+
+
+def test_pack_rejections(kv):
+    s = synth.SHAPES["tiny"]
+    cache = _FakeCache(kv, s, 12)
+    page = synth.kv_page_bytes(s)
+    wire = _FakeBuf(3 * s.n_layers * 2 * page)
+    assert _status(kv.kv_pack_blocks, cache, [1, 12, 3], wire, stream=0) == O.ERR_BLOCK_RANGE
+    assert _status(kv.kv_pack_blocks, cache, [1, 2, 3, 4], wire, stream=0) == O.ERR_WIRE_SIZE
+    assert _status(kv.kv_pack_blocks, cache, [1, 2, 3], _FakeBuf(1 << 20, 0x7100000008), stream=0) == O.ERR_ARG
+    assert _status(kv.kv_pack_blocks, cache, [1, 2], wire, wire_layout=5, stream=0) == O.ERR_ARG
+    assert _status(kv.kv_unpack_blocks_batched, cache, [0, 2, 3], [4, 5, 4], [wire, wire], stream=0) == O.ERR_BLOCK_ALIAS
+
+
+def test_prefill_and_decode_rejections(kv):
+    s = synth.SHAPES["tiny"]
+    lib = kv.load()
+    from paper_2608_16477_b200.binding import ModelDesc, Weights
+    fake = 0x7200000000
+    arr = (C.c_void_p * s.n_layers)(*[fake] * s.n_layers)
+    parr = C.cast(arr, C.POINTER(C.c_void_p))
+    w = Weights(fake, fake, fake, parr, parr, parr, parr, parr, parr)
+    d = ModelDesc(s.n_layers, s.hidden, s.n_q_heads, s.n_kv_heads, s.head_dim, s.ffn, s.vocab, 1e6, 1e-6)
+    h = C.c_void_p()
+    assert lib.kv_model_create(C.byref(d), C.byref(w), C.byref(h)) == 0
+    bad = ModelDesc(s.n_layers, s.hidden, 3, 2, s.head_dim, s.ffn, s.vocab, 1e6, 1e-6)
+    h2 = C.c_void_p()
+    assert lib.kv_model_create(C.byref(bad), C.byref(w), C.byref(h2)) == O.ERR_SHAPE
+
+    class M:
+        handle = h
+    need = kv.kv_workspace_bytes(M, kv.KV_OP_PREFILL, 64)
+    assert need > 64 * s.hidden * 4
+    cache = _FakeCache(kv, s, 12)
+    ws = _FakeBuf(need, 0x7300000000)
+    ids = list(range(64))
+    table = [3, 1, 4, 5]
+
+    def prefill(ids=ids, table=table, pos0=0, ws=ws, cache=cache):
+        return _status(kv.kv_prefill_prefix, M, cache, ids, table, pos0=pos0, workspace=ws, stream=0)
+    assert prefill(ids=ids[:63] + [s.vocab]) == O.ERR_TOKEN_RANGE
+    assert prefill(table=[3, 1, 4]) == O.ERR_TABLE_SHORT
+    assert prefill(table=[3, 1, 4, 12]) == O.ERR_BLOCK_RANGE
+    assert prefill(table=[3, 1, 4, 3]) == O.ERR_BLOCK_ALIAS
+    assert prefill(pos0=8, table=table + [6]) == O.ERR_SPLIT_UNALIGNED
+    assert prefill(ws=_FakeBuf(need - 1, 0x7300000000)) == O.ERR_WORKSPACE
+    assert prefill(ws=_FakeBuf(need, 0x7300000010)) == O.ERR_WORKSPACE
+    wide = synth.ModelShape(**{**s.__dict__, "n_kv_heads": 4})
+    assert prefill(cache=_FakeCache(kv, wide, 12)) == O.ERR_SHAPE
+    dneed = kv.kv_workspace_bytes(M, kv.KV_OP_DECODE, 64)
+    dws = _FakeBuf(dneed, 0x7300000000)
+    logits = _FakeBuf(4 * s.vocab, 0x7400000000)
+    assert _status(kv.kv_decode_step, M, cache, 5, 63, [3, 1, 4], logits, workspace=dws, stream=0) == O.ERR_TABLE_SHORT
+    assert _status(kv.kv_decode_step, M, cache, s.vocab, 63, table, logits, workspace=dws, stream=0) == O.ERR_TOKEN_RANGE
+    lib.kv_model_destroy(h)

@@ -374,3 +374,26 @@ def test_write_read_kv_through_block_table():
     assert np.array_equal(k2, O.from_bf16_bits(O.to_bf16_bits(K)))
     assert np.array_equal(v2, O.from_bf16_bits(O.to_bf16_bits(V)))
     assert not c[:, :, [1, 2, 4, 5, 7]].any()
+
+
+def test_bf16_storage_points_only_round():
+    """The bf16-storage variant is the same function with roundings inserted: its K/V are exactly
+    bf16-representable, it stays within a few bf16 ulps of the exact path, and on inputs where every
+    stored tensor is already representable it changes nothing."""
+    s = synth.SHAPES["tiny"]
+    head = synth.head_weights(s, 0)
+    lw = [synth.layer_weights(s, 0, l) for l in range(s.n_layers)]
+    ids = synth.token_ids(s, 0, 48)
+    K0, V0, l0 = O.forward_full(s, head, lambda l: lw[l], ids)
+    K1, V1, l1 = O.forward_full(s, head, lambda l: lw[l], ids, act_bf16=True)
+    assert np.array_equal(K1, O.from_bf16_bits(O.to_bf16_bits(K1))) and np.array_equal(V1, O.from_bf16_bits(O.to_bf16_bits(V1)))
+    assert 0 < np.max(np.abs(K1 - K0)) < 2e-2 and np.sqrt(np.sum((l1 - l0) ** 2) / np.sum(l0 ** 2)) < 1e-2
+    # powers of two everywhere: nothing to round
+    t = synth.ModelShape("t", n_layers=1, hidden=4, n_q_heads=1, n_kv_heads=1, head_dim=4, ffn=4, vocab=3, rms_eps=0.0)
+    eye = np.eye(4)
+    w = {"attn_norm": np.ones(4), "ffn_norm": np.ones(4), "w_qkv": np.vstack([eye, eye, eye]), "w_o": eye,
+         "w_gate_up": np.vstack([eye, eye]), "w_down": eye}
+    x = np.array([[2.0, -2.0, 2.0, -2.0]])
+    a = O.layer_forward(t, w, x, np.array([0]), skip_after_kv=True)
+    b = O.layer_forward(t, w, x, np.array([0]), skip_after_kv=True, act_bf16=True)
+    assert np.array_equal(a[1], b[1]) and np.array_equal(a[2], b[2])
