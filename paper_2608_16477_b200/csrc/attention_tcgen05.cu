@@ -1,0 +1,349 @@
+// Causal GQA flash attention for prefill on the 5th-generation tensor cores (pos0 = 0, head_dim 64 or 128).
+//
+// One CTA works on ONE 128-row query tile of TWO query heads that share a KV head (tiles "a" and "b"), so
+// every K/V tile fetched by TMA feeds both, and the two softmax warpgroups alternate with the tensor core:
+// while one tile's scores are being exponentiated, the other tile's MMAs run.
+//
+//   warp 0      TMA producer: Q tiles once, then K and V tiles (128 keys) into a 2-stage ring.
+//   warp 1      TMEM allocation and MMA issue:  S = Q K^T  (both operands K-major in shared memory),
+//               O += P V  (P read from TMEM, V as an MN-major shared-memory operand: no transposes).
+//   warps 4-7   softmax of tile a, warps 8-11 softmax of tile b: one thread per query row (= TMEM lane).
+//               Pass 1 reads the row of S for its maximum, pass 2 turns it into bf16 probabilities written
+//               back over the first half of S in TMEM.  Statistics stay in fp32; the running maximum is
+//               only advanced (and O rescaled in TMEM) when it grows by more than 8 in the log2 domain,
+//               which keeps exp2 arguments <= 8 and makes rescaling rare.
+// TMEM columns: S_a [0,128)  S_b [128,256)  O_a [256,256+D)  O_b [384,384+D).
+// Tiles are launched heaviest-first (causal work grows with the row tile index).
+// Every mbarrier wait is bounded; a wait that runs out is recorded in the status block and the CTA drains.
+#include "tc_common.cuh"
+
+namespace kvr {
+
+namespace {
+
+constexpr int kBM = 128;            // query rows per tile
+constexpr int kBN = 128;            // keys per KV tile
+constexpr int kKvStages = 2;
+constexpr int kAttnThreads = 384;   // 12 warps
+constexpr uint32_t kTmemS0 = 0, kTmemS1 = 128, kTmemO0 = 256, kTmemO1 = 384;
+constexpr float kRescaleThreshold = 8.0f;
+
+enum AttnTag { ATAG_Q = 11, ATAG_KV_EMPTY = 12, ATAG_K = 13, ATAG_V = 14, ATAG_S = 15, ATAG_P = 16, ATAG_O = 17 };
+
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+
+// MN-major shared-memory operand (V: keys are the K dimension, head dims contiguous), 128-byte swizzle:
+// 8-key groups are 1024 bytes apart (stride byte offset), 64-dim column blocks `lbo_bytes` apart.
+__device__ __forceinline__ uint64_t umma_desc_mn128(uint32_t smem_addr, uint32_t lbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);
+  d |= (uint64_t)(lbo_bytes >> 4) << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t *>(&h);
+}
+
+template <int D>
+struct AttnSmem {
+  static constexpr int kTileBytes = kBM * D * 2;                 // one Q, K or V tile
+  static constexpr int kQOff = 0;                                // 2 Q tiles
+  static constexpr int kKvOff = 2 * kTileBytes;                  // stages of (K, V)
+  static constexpr int kBarOff = kKvOff + kKvStages * 2 * kTileBytes;
+  static constexpr int kBytes = kBarOff + 256 + 1024;            // barriers + alignment slack
+};
+
+template <int D>
+__global__ void __launch_bounds__(kAttnThreads, 1)
+attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_tokens, int n_q_heads, int n_kv_heads,
+                            float scale_log2, bf16 *__restrict__ out, DeviceStatus *status) {
+  using L = AttnSmem<D>;
+  constexpr int kAtoms = D / 64;                   // 64-column (128-byte) boxes per tile row
+  constexpr int kBoxBytes = kBM * 128;             // one 128-row x 64-col box
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t *smem_gen = smem_raw + (smem_base - tc::smem_u32(smem_raw));
+  const uint32_t bar_base = smem_base + L::kBarOff;
+  // barriers: q_full[2] k_full[2] v_full[2] kv_empty[2] s_full[2] p_ready[2] o_full[2]
+  auto bar = [&](int group, int idx) { return bar_base + 8u * (group * 2 + idx); };
+  enum { B_Q = 0, B_K = 1, B_V = 2, B_KV_EMPTY = 3, B_S = 4, B_P = 5, B_O = 6 };
+  uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(smem_gen + L::kBarOff + 8 * 14);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int group = n_q_heads / n_kv_heads;
+  const int pairs = n_q_heads / 2;
+  const int m_tiles = (n_tokens + kBM - 1) / kBM;
+  const int m_tile = m_tiles - 1 - (int)(blockIdx.x / pairs);     // heaviest row tiles first
+  const int pair = blockIdx.x % pairs;
+  const int head_a = 2 * pair, head_b = head_a + 1;
+  const int kv_head = head_a / group;
+  const int m0 = m_tile * kBM;
+  const int n_kv = m_tile + 1;                                     // causal: key tiles 0 .. m_tile
+  const int q_col[2] = {head_a * D, head_b * D};
+  const int k_col = (n_q_heads + kv_head) * D;
+  const int v_col = (n_q_heads + n_kv_heads + kv_head) * D;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 2; ++i) {
+      tc::mbar_init(bar(B_Q, i), 1);
+      tc::mbar_init(bar(B_K, i), 1);
+      tc::mbar_init(bar(B_V, i), 1);
+      tc::mbar_init(bar(B_KV_EMPTY, i), 1);
+      tc::mbar_init(bar(B_S, i), 1);
+      tc::mbar_init(bar(B_P, i), 128);
+      tc::mbar_init(bar(B_O, i), 1);
+    }
+    *abort_flag = 0;
+    tc::fence_barrier_init();
+  }
+  if (warp == 1) tc::tmem_alloc(tc::smem_u32(tmem_holder), 512);
+  tc::tc_fence_before();
+  __syncthreads();
+  tc::tc_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      tc::tma_prefetch_desc(&tma_qkv);
+      for (int t = 0; t < 2; ++t) {
+        tc::mbar_expect_tx(bar(B_Q, t), L::kTileBytes);
+        for (int a = 0; a < kAtoms; ++a)
+          tc::tma_load_2d(smem_base + L::kQOff + t * L::kTileBytes + a * kBoxBytes, &tma_qkv, q_col[t] + a * 64, m0,
+                          bar(B_Q, t));
+      }
+      for (int j = 0; j < n_kv; ++j) {
+        const int st = j & 1;
+        const uint32_t ph = (j >> 1) & 1;
+        if (!tc::mbar_wait(bar(B_KV_EMPTY, st), ph ^ 1, abort_flag, status, ATAG_KV_EMPTY)) break;
+        const uint32_t k_s = smem_base + L::kKvOff + st * 2 * L::kTileBytes;
+        const uint32_t v_s = k_s + L::kTileBytes;
+        tc::mbar_expect_tx(bar(B_K, st), L::kTileBytes);
+        for (int a = 0; a < kAtoms; ++a)
+          tc::tma_load_2d(k_s + a * kBoxBytes, &tma_qkv, k_col + a * 64, j * kBN, bar(B_K, st));
+        tc::mbar_expect_tx(bar(B_V, st), L::kTileBytes);
+        for (int a = 0; a < kAtoms; ++a)
+          tc::tma_load_2d(v_s + a * kBoxBytes, &tma_qkv, v_col + a * 64, j * kBN, bar(B_V, st));
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = tc::umma_idesc_bf16(kBM, kBN);
+      constexpr uint32_t idesc_pv = tc::umma_idesc_bf16(kBM, D) | (1u << 16);   // B (= V) is MN-major
+      const uint32_t s_tmem[2] = {tmem_base + kTmemS0, tmem_base + kTmemS1};
+      const uint32_t o_tmem[2] = {tmem_base + kTmemO0, tmem_base + kTmemO1};
+      auto issue_qk = [&](int t, int st) {
+        const uint32_t q_s = smem_base + L::kQOff + t * L::kTileBytes;
+        const uint32_t k_s = smem_base + L::kKvOff + st * 2 * L::kTileBytes;
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+          const uint32_t off = (ks / 4) * kBoxBytes + (ks % 4) * 32;
+          tc::umma_bf16(s_tmem[t], tc::umma_desc_k128(q_s + off), tc::umma_desc_k128(k_s + off), idesc_qk, ks != 0);
+        }
+        tc::umma_commit(bar(B_S, t));
+      };
+      bool ok = tc::mbar_wait(bar(B_Q, 0), 0, abort_flag, status, ATAG_Q) &&
+                tc::mbar_wait(bar(B_Q, 1), 0, abort_flag, status, ATAG_Q) &&
+                tc::mbar_wait(bar(B_K, 0), 0, abort_flag, status, ATAG_K);
+      if (ok) {
+        tc::tc_fence_after();
+        issue_qk(0, 0);
+        issue_qk(1, 0);
+      }
+      for (int j = 0; j < n_kv && ok; ++j) {
+        const int st = j & 1;
+        const uint32_t ph = (j >> 1) & 1;
+        const uint32_t v_s = smem_base + L::kKvOff + st * 2 * L::kTileBytes + L::kTileBytes;
+        for (int t = 0; t < 2 && ok; ++t) {
+          ok = tc::mbar_wait(bar(B_P, t), j & 1, abort_flag, status, ATAG_P) &&
+               tc::mbar_wait(bar(B_V, st), ph, abort_flag, status, ATAG_V);
+          if (!ok) break;
+          tc::tc_fence_after();
+#pragma unroll
+          for (int ks = 0; ks < kBN / 16; ++ks)   // 16 keys per slice: 8 TMEM columns of P, 2048 bytes of V
+            tc::umma_bf16_ts(o_tmem[t], s_tmem[t] + ks * 8, umma_desc_mn128(v_s + ks * 2048, kBoxBytes), idesc_pv,
+                             (j | ks) != 0);
+          if (t == 1) tc::umma_commit(bar(B_KV_EMPTY, st));
+          if (j + 1 < n_kv) {
+            ok = tc::mbar_wait(bar(B_K, st ^ 1), ((j + 1) >> 1) & 1, abort_flag, status, ATAG_K);
+            if (!ok) break;
+            tc::tc_fence_after();
+            issue_qk(t, st ^ 1);
+          } else {
+            tc::umma_commit(bar(B_O, t));
+          }
+        }
+      }
+    }
+  } else if (warp >= 4) {
+    // ---------------------------------------------------------------- softmax warpgroups
+    const int t = (warp - 4) >> 2;                 // 0: tile a, 1: tile b
+    const int quarter = warp & 3;
+    const int row_in_tile = quarter * 32 + lane;
+    const int qi = m0 + row_in_tile;               // absolute query position (pos0 = 0)
+    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+    const uint32_t s_t = tmem_base + lane_base + (t == 0 ? kTmemS0 : kTmemS1);
+    const uint32_t o_t = tmem_base + lane_base + (t == 0 ? kTmemO0 : kTmemO1);
+    float m_ref = -INFINITY, l_sum = 0.f;
+    bool ok = true;
+    for (int j = 0; j < n_kv; ++j) {
+      ok = tc::mbar_wait(bar(B_S, t), j & 1, abort_flag, status, ATAG_S);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc::tc_fence_after();
+      const bool diag = (j == n_kv - 1);
+      const int limit = qi - j * kBN;              // keys with column > limit are masked
+      // pass 1: row maximum
+      float mx = -INFINITY;
+#pragma unroll 1
+      for (int c = 0; c < kBN / 32; ++c) {
+        uint32_t r[32];
+        tc::tmem_ld32(s_t + c * 32, r);
+        tc::tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const float s = __uint_as_float(r[i]);
+          if (!diag || c * 32 + i <= limit) mx = fmaxf(mx, s);
+        }
+      }
+      mx *= scale_log2;
+      bool rescale = false;
+      float factor = 1.f;
+      if (j == 0) {
+        m_ref = mx;
+      } else if (mx > m_ref + kRescaleThreshold) {
+        rescale = true;
+        factor = exp2f(m_ref - mx);
+        m_ref = mx;
+        l_sum *= factor;
+      }
+      if (__any_sync(0xffffffffu, rescale)) {
+        // O of this tile is idle: the MMAs that produced S_j were issued after PV_{j-1}
+#pragma unroll 1
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t r[32];
+          tc::tmem_ld32(o_t + c * 32, r);
+          tc::tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * factor);
+          tmem_st32(o_t + c * 32, r);
+        }
+      }
+      // pass 2: probabilities, written over S as packed bf16 (two keys per 32-bit column)
+#pragma unroll 1
+      for (int c = 0; c < kBN / 32; ++c) {
+        uint32_t r[32];
+        tc::tmem_ld32(s_t + c * 32, r);
+        tc::tmem_ld_wait();
+        uint32_t pk[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          float p0 = exp2f(__uint_as_float(r[2 * i]) * scale_log2 - m_ref);
+          float p1 = exp2f(__uint_as_float(r[2 * i + 1]) * scale_log2 - m_ref);
+          if (diag) {
+            if (c * 32 + 2 * i > limit) p0 = 0.f;
+            if (c * 32 + 2 * i + 1 > limit) p1 = 0.f;
+          }
+          l_sum += p0 + p1;
+          pk[i] = pack2(p0, p1);
+        }
+        tmem_st16(s_t + c * 16, pk);
+      }
+      tc::tmem_st_wait();
+      tc::tc_fence_before();
+      tc::mbar_arrive(bar(B_P, t));
+    }
+    if (ok) {
+      ok = tc::mbar_wait(bar(B_O, t), 0, abort_flag, status, ATAG_O);
+      ok = __all_sync(0xffffffffu, ok);
+    }
+    if (ok) {
+      tc::tc_fence_after();
+      const float inv = 1.f / l_sum;
+      const int head = (t == 0) ? head_a : head_b;
+      bf16 *orow = out + (long long)qi * n_q_heads * D + head * D;
+#pragma unroll 1
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t r[32];
+        tc::tmem_ld32(o_t + c * 32, r);
+        tc::tmem_ld_wait();
+        if (qi < n_tokens) {
+          uint4 *dst = reinterpret_cast<uint4 *>(orow + c * 32);
+#pragma unroll
+          for (int v = 0; v < 4; ++v)
+            dst[v] = make_uint4(pack2(__uint_as_float(r[8 * v]) * inv, __uint_as_float(r[8 * v + 1]) * inv),
+                                pack2(__uint_as_float(r[8 * v + 2]) * inv, __uint_as_float(r[8 * v + 3]) * inv),
+                                pack2(__uint_as_float(r[8 * v + 4]) * inv, __uint_as_float(r[8 * v + 5]) * inv),
+                                pack2(__uint_as_float(r[8 * v + 6]) * inv, __uint_as_float(r[8 * v + 7]) * inv));
+        }
+      }
+    }
+  }
+
+  tc::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc::tc_fence_after();
+    tc::tmem_dealloc(tmem_base, 512);
+  }
+}
+
+}  // namespace
+
+// pos0 == 0, head_dim 64 or 128, even number of query heads per KV head.
+int attention_prefill_tc(const bf16 *qkv, int n_tokens, int n_q_heads, int n_kv_heads, int head_dim, bf16 *out,
+                         int *status_dev, cudaStream_t st) {
+  if (n_tokens <= 0) return KV_OK;
+  const int qkv_dim = (n_q_heads + 2 * n_kv_heads) * head_dim;
+  CUtensorMap map;
+  int rc = tc::make_tmap_2d(&map, qkv, n_tokens, qkv_dim, qkv_dim, kBM);
+  if (rc != KV_OK) return rc;
+  static bool attr_set = false;
+  if (!attr_set) {
+    KV_CUDA(cudaFuncSetAttribute(attention_prefill_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 AttnSmem<64>::kBytes));
+    KV_CUDA(cudaFuncSetAttribute(attention_prefill_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 AttnSmem<128>::kBytes));
+    attr_set = true;
+  }
+  const int m_tiles = (n_tokens + kBM - 1) / kBM;
+  const int grid = m_tiles * (n_q_heads / 2);
+  const float scale_log2 = 1.4426950408889634f / sqrtf((float)head_dim);
+  DeviceStatus *status = reinterpret_cast<DeviceStatus *>(status_dev);
+  if (head_dim == 64)
+    attention_prefill_tc_kernel<64><<<grid, kAttnThreads, AttnSmem<64>::kBytes, st>>>(map, n_tokens, n_q_heads,
+                                                                                     n_kv_heads, scale_log2, out, status);
+  else
+    attention_prefill_tc_kernel<128><<<grid, kAttnThreads, AttnSmem<128>::kBytes, st>>>(map, n_tokens, n_q_heads,
+                                                                                       n_kv_heads, scale_log2, out, status);
+  KV_COUNT_LAUNCH();
+  KV_CUDA(cudaGetLastError());
+  return KV_OK;
+}
+
+}  // namespace kvr

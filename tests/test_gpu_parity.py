@@ -174,7 +174,8 @@ def test_rmsnorm_rows(kv, torch):
     assert np.all(np.abs(got - want) <= 2.0 ** -8 * np.abs(want) + 1e-6)
 
 
-@pytest.mark.parametrize("t,hq,hkv,d", [(70, 4, 2, 64), (200, 8, 1, 128), (129, 2, 2, 128)])
+@pytest.mark.parametrize("t,hq,hkv,d", [(70, 4, 2, 64), (200, 8, 1, 128), (129, 2, 2, 128), (1000, 4, 2, 128),
+                                      (384, 8, 2, 64), (128, 2, 1, 128), (1, 2, 1, 64)])
 def test_attention_prefill_kernel(kv, torch, t, hq, hkv, d):
     rng = np.random.default_rng(7 + t)
     qkv = synth.bf16_round_f32(rng.standard_normal((t, (hq + 2 * hkv) * d), dtype=np.float32))
@@ -276,8 +277,10 @@ def test_scenario_wide_reduced_depth(kv, name, layers, k, n):
         st = error_stats(got, ref)
         report["bf16pt_" + nm] = st
         assert st["rel_l2"] <= 5e-3, (nm, st)                      # half the stated bound
-        # element-wise: a few bf16 ulps (one ulp is at most 2^-7 of the value)
-        assert np.all(np.abs(got - ref) <= np.maximum(2e-2, 2.0 ** -6 * np.abs(ref))), (nm, st)
+        # element-wise: the rel-L2 bound caps the error's standard deviation at 5e-3 * rms(ref); 8 sigma
+        # covers ~1e9 roughly Gaussian samples, plus one bf16 ulp of the value itself (at most 2^-7 |ref|)
+        rms = float(np.sqrt(np.mean(np.asarray(ref, dtype=np.float64) ** 2)))
+        assert np.all(np.abs(got - ref) <= 8 * 5e-3 * rms + 2.0 ** -7 * np.abs(ref)), (nm, st)
     Kref, Vref, logits_ref = oracle_reference(s, 0, ids)
     for nm, got, ref in (("K", res["K"], Kref), ("V", res["V"], Vref)):
         st = error_stats(got, ref)
