@@ -1,0 +1,102 @@
+"""Runs ONE kernel of the hot path a few times at the benchmark's shapes, for profiler captures.
+
+  python -m paper_2608_16477_b200.profile_case gemm_gate_up [--tokens 4096] [--iters 3]
+  cases: gemm_qkv, gemm_o, gemm_gate_up, gemm_down, attention, pack, unpack, decode_gemv
+
+Inputs are synthetic and larger than L2 where the kernel is bandwidth-bound; a few GB at most are held on
+the device so a multi-pass capture stays short.  Prints the CUDA-event time per launch.
+"""
+import argparse
+import sys
+
+import numpy as np
+
+import synth
+
+
+def main():
+    import torch
+    import paper_2608_16477_b200 as kv
+    ap = argparse.ArgumentParser()
+    ap.add_argument("case")
+    ap.add_argument("--shape", default="32b")
+    ap.add_argument("--tokens", type=int, default=4096)
+    ap.add_argument("--iters", type=int, default=3)
+    ap.add_argument("--blocks", type=int, default=32, help="pack/unpack: blocks per launch")
+    a = ap.parse_args()
+    kv.load()
+    s = synth.SHAPES[a.shape]
+    t = a.tokens
+    dev = "cuda"
+    g = torch.Generator(device=dev).manual_seed(0)
+
+    def rnd(*shape, std=1.0):
+        return torch.empty(*shape, dtype=torch.bfloat16, device=dev).normal_(0.0, std, generator=g)
+    status = torch.zeros(64, dtype=torch.int32, device=dev)
+    if a.case.startswith("gemm"):
+        if a.case == "gemm_gate_up":
+            x, w, mode = rnd(t, s.hidden), rnd(2 * s.ffn, s.hidden, std=0.02), 2
+            out, resid, flops = torch.empty(t, s.ffn, dtype=torch.bfloat16, device=dev), None, 2.0 * t * s.hidden * 2 * s.ffn
+        elif a.case == "gemm_down":
+            x, w, mode = rnd(t, s.ffn), rnd(s.hidden, s.ffn, std=0.02), 1
+            out, resid, flops = None, torch.zeros(t, s.hidden, dtype=torch.float32, device=dev), 2.0 * t * s.hidden * s.ffn
+        elif a.case == "gemm_o":
+            x, w, mode = rnd(t, s.q_dim), rnd(s.hidden, s.q_dim, std=0.02), 1
+            out, resid, flops = None, torch.zeros(t, s.hidden, dtype=torch.float32, device=dev), 2.0 * t * s.hidden * s.q_dim
+        elif a.case == "gemm_qkv":
+            x, w, mode = rnd(t, s.hidden), rnd(s.qkv_dim, s.hidden, std=0.02), 0
+            out, resid, flops = torch.empty(t, s.qkv_dim, dtype=torch.bfloat16, device=dev), None, 2.0 * t * s.hidden * s.qkv_dim
+        else:
+            raise SystemExit(f"unknown case {a.case}")
+        run = lambda: kv.kv_op_gemm(x, w, mode, out=out, resid=resid, status=status)
+        work, unit = flops / 1e12, "TFLOP/s"
+    elif a.case == "attention":
+        qkv = rnd(t, s.qkv_dim)
+        out = torch.empty(t, s.q_dim, dtype=torch.bfloat16, device=dev)
+        run = lambda: kv.kv_op_attention_prefill(qkv, s.n_q_heads, s.n_kv_heads, s.head_dim, out, status=status)
+        work, unit = 2.0 * s.n_q_heads * s.head_dim * t * (t + 1) / 1e12, "TFLOP/s"
+    elif a.case in ("pack", "unpack"):
+        pool = 1024                                   # 4 GiB pool at the 32B shape
+        cache = kv.PagedCache(s, pool)
+        kv.kv_fill_pattern(cache.data, cache.data.numel() * 2, seed=1)
+        perm = synth.block_permutation(1, pool)
+        n_sets = 4
+        wires = [torch.empty(a.blocks * s.n_layers * 2 * cache.page_bytes, dtype=torch.uint8, device=dev)
+                 for _ in range(n_sets)]
+        state = {"i": 0}
+
+        def run():
+            i = state["i"] % n_sets
+            state["i"] += 1
+            ids = perm[i * a.blocks:(i + 1) * a.blocks]
+            if a.case == "pack":
+                kv.kv_pack_blocks(cache, ids, wires[i])
+            else:
+                kv.kv_unpack_assemble(cache, wires[i], np.arange(a.blocks), ids, [], a.blocks * s.block_size)
+        work, unit = 2.0 * a.blocks * s.n_layers * 2 * cache.page_bytes / 1e9, "GB/s"
+    elif a.case == "decode_gemv":
+        w = rnd(2 * s.ffn, s.hidden, std=0.02)
+        x = torch.randn(s.hidden, device=dev)
+        y = torch.empty(s.ffn, device=dev)
+        lib = kv.load()
+        raise SystemExit("decode_gemv has no single-kernel entry point; profile bench.py instead")
+    else:
+        raise SystemExit(f"unknown case {a.case}")
+    run()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(a.iters):
+        run()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / a.iters
+    if int(status[0]) != 0:
+        raise SystemExit(f"device wait ran out: {status[:8].tolist()}")
+    per = work / (ms * 1e-3)
+    print(f"{a.case}: {ms * 1e3:.1f} us per launch, {per:.1f} {unit}")
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())
