@@ -28,7 +28,7 @@
  * fused QKV projection (rows ordered Q | K | V, heads contiguous), rotate-half RoPE, causal
  * grouped-query attention (query head h reads KV head h / (Hq/Hkv)), output projection, RMSNorm,
  * SwiGLU FFN (rows of w_gate_up ordered gate | up), final RMSNorm and LM head.
- * All matrices are row-major [out, in]; y = x W^T.
+ * All matrices are row-major [out, in]; y = x W^T.  head_dim must be 64 or 128, hidden and ffn multiples of 8.
  *
  * Paged cache: page(layer, kv, block) is block_size * n_kv_heads * head_dim contiguous bf16,
  * laid out [slot][kv_head][dim], at base + layer*layer_stride + kv*kv_stride + block*block_stride

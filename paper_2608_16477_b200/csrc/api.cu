@@ -239,7 +239,7 @@ int32_t kv_model_create(const kv_model_desc *desc, const kv_weights *w, kv_model
   if (d.n_layers <= 0 || d.hidden <= 0 || d.n_q_heads <= 0 || d.n_kv_heads <= 0 || d.head_dim <= 0 || d.ffn <= 0 ||
       d.vocab <= 0)
     return KV_ERR_ARG;
-  if (d.n_q_heads % d.n_kv_heads != 0 || (d.head_dim != 64 && d.head_dim != 128 && d.head_dim != 256) || d.hidden % 8 != 0 ||
+  if (d.n_q_heads % d.n_kv_heads != 0 || (d.head_dim != 64 && d.head_dim != 128) || d.hidden % 8 != 0 ||
       d.ffn % 8 != 0)
     return KV_ERR_SHAPE;
   if (!w->embed_dev || !w->lm_head_dev || !w->final_norm_dev || !w->attn_norm_dev || !w->w_qkv_dev || !w->w_o_dev ||
@@ -578,8 +578,8 @@ int32_t kv_op_paged_attention(const float *q_dev, int32_t n_q_heads, const kv_ca
     return KV_ERR_ARG;
   int rc = check_cache(cache);
   if (rc != KV_OK) return rc;
-  if (layer < 0 || layer >= cache->n_layers || n_q_heads % cache->n_kv_heads != 0 || cache->head_dim % 32 != 0 ||
-      cache->head_dim > 256)
+  if (layer < 0 || layer >= cache->n_layers || n_q_heads % cache->n_kv_heads != 0 ||
+      (cache->head_dim != 64 && cache->head_dim != 128))
     return KV_ERR_SHAPE;
   if (scratch_bytes < paged_attention_scratch_bytes(n_q_heads, cache->head_dim, n_ctx)) return KV_ERR_WORKSPACE;
   return paged_attention(q_dev, n_q_heads, make_view(cache), layer, block_table_dev, n_ctx, scratch_dev, out_dev,

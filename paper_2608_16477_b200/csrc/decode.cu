@@ -104,12 +104,20 @@ int gemv(const bf16 *w, const float *x, int n, int k, int mode, float *y, cudaSt
   return KV_OK;
 }
 
-// Rotate the Q and K heads of the fp32 qkv vector in place (angles in fp64) and append K/V (bf16) to the cache.
+// Rotate the Q and K heads of the fp32 qkv vector in place and append K/V (bf16) to the cache.
+// The d/2 angles pos * base^(-2j/d) are formed once in fp64 (one thread per frequency) and shared.
 __global__ void __launch_bounds__(256) rope_store_kv_one_kernel(float *__restrict__ qkv, int pos, int n_q_heads,
                                                                 int n_kv_heads, int head_dim, float base,
                                                                 CacheView cache, int layer,
                                                                 const int *__restrict__ block_table) {
+  __shared__ float2 cs[128];
   const int half = head_dim / 2;
+  for (int j = threadIdx.x; j < half; j += blockDim.x) {
+    double s, c;
+    sincos((double)pos * pow((double)base, -(double)j / (double)half), &s, &c);
+    cs[j] = make_float2((float)c, (float)s);
+  }
+  __syncthreads();
   const int block = block_table[pos / cache.block_size];
   const int slot = pos % cache.block_size;
   bf16 *kpage = reinterpret_cast<bf16 *>(cache.page(layer, 0, block)) + (long long)slot * n_kv_heads * head_dim;
@@ -117,11 +125,10 @@ __global__ void __launch_bounds__(256) rope_store_kv_one_kernel(float *__restric
   const int n_rot = (n_q_heads + n_kv_heads) * half;
   for (int idx = threadIdx.x; idx < n_rot; idx += blockDim.x) {
     const int head = idx / half, j = idx - head * half;
-    double s, c;
-    sincos((double)pos * pow((double)base, -(double)j / (double)half), &s, &c);
+    const float2 c = cs[j];
     float *h = qkv + head * head_dim;
     const float a = h[j], b = h[j + half];
-    const float ra = a * (float)c - b * (float)s, rb = b * (float)c + a * (float)s;
+    const float ra = a * c.x - b * c.y, rb = b * c.x + a * c.y;
     h[j] = ra;
     h[j + half] = rb;
     if (head >= n_q_heads) {
@@ -145,9 +152,15 @@ int rope_store_kv_one(float *qkv, int pos, int n_q_heads, int n_kv_heads, int he
 
 // ---- paged decode attention ---------------------------------------------------------------
 // Partial record per (q head, split): m, l, acc[d].
-constexpr int kPaWarps = 4;
-constexpr int kPaSplitKeys = 256;   // keys per split (multiple of any block size in use)
-constexpr int kPaMaxDimsPerLane = 8;  // head_dim <= 256
+// One CTA of 256 threads per (KV head, 256-key split), serving every query head of the group so each K/V
+// row is read from HBM once:
+//   phase 1  thread t loads the whole K row of key t (16-byte loads, all in flight at once) and scores it
+//            against the group's queries held in shared memory;
+//   phase 2  one warp per head: maximum, exponentials and their sum over the split's scores;
+//   phase 3  warp w walks keys 32w..32w+31, each lane owning d/32 dims of V, accumulating p * v for all
+//            heads; the eight warps' partial sums meet in shared memory.
+constexpr int kPaSplitKeys = 256;   // keys per split = threads per CTA
+constexpr int kPaHeadChunk = 8;     // query heads handled per pass over the keys
 
 static int pa_splits(int n_ctx) {
   int s = (n_ctx + kPaSplitKeys - 1) / kPaSplitKeys;
@@ -158,63 +171,167 @@ long long paged_attention_scratch_bytes(int n_q_heads, int head_dim, int n_ctx) 
   return (long long)n_q_heads * pa_splits(n_ctx) * (head_dim + 2) * (long long)sizeof(float);
 }
 
-__global__ void __launch_bounds__(kPaWarps * 32) paged_attention_split_kernel(
+// DPL consecutive bf16 -> fp32 with one vector load (the address is DPL*2-byte aligned)
+template <int DPL>
+__device__ __forceinline__ void load_bf16(const bf16 *p, float (&out)[DPL]) {
+  static_assert(DPL == 2 || DPL == 4 || DPL == 8, "dims per lane");
+  if constexpr (DPL == 8) {
+    const uint4 raw = *reinterpret_cast<const uint4 *>(p);
+    const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 f = __bfloat1622float2(h[i]);
+      out[2 * i] = f.x;
+      out[2 * i + 1] = f.y;
+    }
+  } else if constexpr (DPL == 4) {
+    const uint2 raw = *reinterpret_cast<const uint2 *>(p);
+    const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+    const float2 a = __bfloat1622float2(h[0]), b = __bfloat1622float2(h[1]);
+    out[0] = a.x; out[1] = a.y; out[2] = b.x; out[3] = b.y;
+  } else {
+    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(p));
+    out[0] = a.x; out[1] = a.y;
+  }
+}
+
+template <int D>
+__global__ void __launch_bounds__(kPaSplitKeys) paged_attention_split_kernel(
     const float *__restrict__ q, int n_q_heads, CacheView cache, int layer, const int *__restrict__ block_table,
     int n_ctx, float *__restrict__ partial) {
-  const int head = blockIdx.x, split = blockIdx.y, n_splits = gridDim.y;
-  const int d = cache.head_dim;
-  const int g = head / (n_q_heads / cache.n_kv_heads);
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int dpl = d / 32;   // dims per lane, lane owns dims lane*dpl .. lane*dpl+dpl-1
-  const float scale = rsqrtf((float)d);
-  float qr[kPaMaxDimsPerLane], acc[kPaMaxDimsPerLane];
-#pragma unroll
-  for (int i = 0; i < kPaMaxDimsPerLane; ++i) {
-    qr[i] = (i < dpl) ? q[head * d + lane * dpl + i] * scale : 0.f;
-    acc[i] = 0.f;
-  }
-  float m = -FLT_MAX, l = 0.f;
+  constexpr int DPL = D / 32;
+  constexpr int HC = kPaHeadChunk;
+  __shared__ __align__(16) float q_s[HC][D];
+  __shared__ float p_s[HC][kPaSplitKeys];
+  __shared__ __align__(16) float red_s[kPaSplitKeys / 32][HC][D];
+  __shared__ float ml_s[HC][2];
+  const int g = blockIdx.x, split = blockIdx.y, n_splits = gridDim.y;
+  const int group = n_q_heads / cache.n_kv_heads;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float scale = rsqrtf((float)D);
   const int j0 = split * kPaSplitKeys;
-  const int j1 = min(n_ctx, j0 + kPaSplitKeys);
-  for (int j = j0 + warp; j < j1; j += kPaWarps) {
-    const int block = block_table[j / cache.block_size];
-    const long long off = ((long long)(j % cache.block_size) * cache.n_kv_heads + g) * d + lane * dpl;
-    const bf16 *kp = reinterpret_cast<const bf16 *>(cache.page(layer, 0, block)) + off;
-    const bf16 *vp = reinterpret_cast<const bf16 *>(cache.page(layer, 1, block)) + off;
-    float s = 0.f;
+  const int n_keys = min(n_ctx - j0, kPaSplitKeys);
+
+  // this thread's key: K row into registers (phase 1 operand), V row address for later
+  const int jk = j0 + min(tid, n_keys - 1);
+  const long long row_off = ((long long)(jk % cache.block_size) * cache.n_kv_heads + g) * D;
+  const int blk_k = block_table[jk / cache.block_size];
+  uint4 kraw[D / 8];
+  {
+    const uint4 *kp = reinterpret_cast<const uint4 *>(reinterpret_cast<const bf16 *>(cache.page(layer, 0, blk_k)) + row_off);
 #pragma unroll
-    for (int i = 0; i < kPaMaxDimsPerLane; ++i)
-      if (i < dpl) s += qr[i] * __bfloat162float(kp[i]);
-    s = warp_sum_d(s);
-    const float mn = fmaxf(m, s);
-    const float corr = __expf(m - mn), p = __expf(s - mn);
-    l = l * corr + p;
-#pragma unroll
-    for (int i = 0; i < kPaMaxDimsPerLane; ++i)
-      if (i < dpl) acc[i] = acc[i] * corr + p * __bfloat162float(vp[i]);
-    m = mn;
+    for (int v = 0; v < D / 8; ++v) kraw[v] = kp[v];
   }
-  // merge the warps of this CTA
-  __shared__ float sm_m[kPaWarps], sm_l[kPaWarps];
-  __shared__ float sm_acc[kPaWarps][256];
-  if (lane == 0) { sm_m[warp] = m; sm_l[warp] = l; }
+
+  for (int h0 = 0; h0 < group; h0 += HC) {
+    const int nh = min(HC, group - h0);
+    __syncthreads();   // previous chunk fully consumed
+    for (int e = tid; e < nh * D; e += kPaSplitKeys)
+      q_s[e / D][e % D] = q[(long long)(g * group + h0 + e / D) * D + e % D] * scale;
+    __syncthreads();
+    // ---- phase 1: scores of this thread's key against nh heads
+    {
+      float sc[HC];
 #pragma unroll
-  for (int i = 0; i < kPaMaxDimsPerLane; ++i)
-    if (i < dpl) sm_acc[warp][lane * dpl + i] = acc[i];
-  __syncthreads();
-  float *rec = partial + ((long long)head * n_splits + split) * (d + 2);
-  float mm = -FLT_MAX;
-  for (int w = 0; w < kPaWarps; ++w) mm = fmaxf(mm, sm_m[w]);
-  if (threadIdx.x == 0) {
-    float ll = 0.f;
-    for (int w = 0; w < kPaWarps; ++w) ll += sm_l[w] * __expf(sm_m[w] - mm);
-    rec[0] = mm;
-    rec[1] = ll;
-  }
-  for (int c = threadIdx.x; c < d; c += blockDim.x) {
-    float a = 0.f;
-    for (int w = 0; w < kPaWarps; ++w) a += sm_acc[w][c] * __expf(sm_m[w] - mm);
-    rec[2 + c] = a;
+      for (int h = 0; h < HC; ++h) sc[h] = 0.f;
+#pragma unroll
+      for (int v = 0; v < D / 8; ++v) {
+        const __nv_bfloat162 *hk = reinterpret_cast<const __nv_bfloat162 *>(&kraw[v]);
+        const float2 k0 = __bfloat1622float2(hk[0]), k1 = __bfloat1622float2(hk[1]);
+        const float2 k2 = __bfloat1622float2(hk[2]), k3 = __bfloat1622float2(hk[3]);
+#pragma unroll
+        for (int h = 0; h < HC; ++h) {
+          if (h < nh) {
+            const float4 qa = *reinterpret_cast<const float4 *>(&q_s[h][v * 8]);
+            const float4 qb = *reinterpret_cast<const float4 *>(&q_s[h][v * 8 + 4]);
+            sc[h] += k0.x * qa.x + k0.y * qa.y + k1.x * qa.z + k1.y * qa.w + k2.x * qb.x + k2.y * qb.y + k3.x * qb.z +
+                     k3.y * qb.w;
+          }
+        }
+      }
+#pragma unroll
+      for (int h = 0; h < HC; ++h)
+        if (h < nh) p_s[h][tid] = (tid < n_keys) ? sc[h] : -FLT_MAX;
+    }
+    __syncthreads();
+    // ---- phase 2: warp h turns the scores of head h into exponentials
+    if (warp < nh) {
+      float v[kPaSplitKeys / 32];
+      float mx = -FLT_MAX;
+#pragma unroll
+      for (int i = 0; i < kPaSplitKeys / 32; ++i) {
+        v[i] = p_s[warp][lane + 32 * i];
+        mx = fmaxf(mx, v[i]);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      float sum = 0.f;
+#pragma unroll
+      for (int i = 0; i < kPaSplitKeys / 32; ++i) {
+        const float e = (lane + 32 * i < n_keys) ? __expf(v[i] - mx) : 0.f;
+        p_s[warp][lane + 32 * i] = e;
+        sum += e;
+      }
+      sum = warp_sum_d(sum);
+      if (lane == 0) {
+        ml_s[warp][0] = mx;
+        ml_s[warp][1] = sum;
+      }
+    }
+    __syncthreads();
+    // ---- phase 3: p * V, warp w over keys 32w .. 32w+31, lane owns DPL dims
+    {
+      float acc[HC][DPL];
+#pragma unroll
+      for (int h = 0; h < HC; ++h)
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) acc[h][i] = 0.f;
+      const int kb = warp * 32;
+      constexpr int U = 8;
+      for (int kk = 0; kk < 32 && kb + kk < n_keys; kk += U) {
+        float vf[U][DPL];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const int j = j0 + min(kb + kk + u, n_keys - 1);
+          const int blk = block_table[j / cache.block_size];
+          const bf16 *vp = reinterpret_cast<const bf16 *>(cache.page(layer, 1, blk)) +
+                           ((long long)(j % cache.block_size) * cache.n_kv_heads + g) * D + lane * DPL;
+          load_bf16<DPL>(vp, vf[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          if (kb + kk + u < n_keys) {
+#pragma unroll
+            for (int h = 0; h < HC; ++h) {
+              if (h < nh) {
+                const float p = p_s[h][kb + kk + u];
+#pragma unroll
+                for (int i = 0; i < DPL; ++i) acc[h][i] += p * vf[u][i];
+              }
+            }
+          }
+        }
+      }
+#pragma unroll
+      for (int h = 0; h < HC; ++h)
+        if (h < nh) {
+#pragma unroll
+          for (int i = 0; i < DPL; ++i) red_s[warp][h][lane * DPL + i] = acc[h][i];
+        }
+    }
+    __syncthreads();
+    for (int e = tid; e < nh * D; e += kPaSplitKeys) {
+      const int h = e / D, c = e % D;
+      float a = 0.f;
+#pragma unroll
+      for (int w = 0; w < kPaSplitKeys / 32; ++w) a += red_s[w][h][c];
+      float *rec = partial + ((long long)(g * group + h0 + h) * n_splits + split) * (D + 2);
+      rec[2 + c] = a;
+      if (c == 0) {
+        rec[0] = ml_s[h][0];
+        rec[1] = ml_s[h][1];
+      }
+    }
   }
 }
 
@@ -236,11 +353,17 @@ __global__ void paged_attention_merge_kernel(const float *__restrict__ partial, 
 int paged_attention(const float *q, int n_q_heads, CacheView cache, int layer, const int *block_table_dev,
                     int n_ctx, void *scratch, float *out, cudaStream_t st) {
   const int splits = pa_splits(n_ctx);
-  paged_attention_split_kernel<<<dim3(n_q_heads, splits), kPaWarps * 32, 0, st>>>(
-      q, n_q_heads, cache, layer, block_table_dev, n_ctx, (float *)scratch);
+  const dim3 grid(cache.n_kv_heads, splits);
+  float *partial = (float *)scratch;
+  if (cache.head_dim == 64)
+    paged_attention_split_kernel<64><<<grid, kPaSplitKeys, 0, st>>>(q, n_q_heads, cache, layer, block_table_dev, n_ctx, partial);
+  else if (cache.head_dim == 128)
+    paged_attention_split_kernel<128><<<grid, kPaSplitKeys, 0, st>>>(q, n_q_heads, cache, layer, block_table_dev, n_ctx, partial);
+  else
+    return KV_ERR_SHAPE;
   KV_COUNT_LAUNCH();
   KV_CUDA(cudaGetLastError());
-  paged_attention_merge_kernel<<<n_q_heads, 128, 0, st>>>((const float *)scratch, splits, cache.head_dim, out);
+  paged_attention_merge_kernel<<<n_q_heads, 128, 0, st>>>(partial, splits, cache.head_dim, out);
   KV_COUNT_LAUNCH();
   KV_CUDA(cudaGetLastError());
   return KV_OK;

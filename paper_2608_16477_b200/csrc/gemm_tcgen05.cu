@@ -24,15 +24,23 @@ namespace kvr {
 namespace {
 
 constexpr int BM = 128;
-constexpr int BN = 256;      // accumulator columns per tile
 constexpr int BK = 64;       // 128 bytes of bf16: one swizzle atom
-constexpr int kStages = 4;
 constexpr int kABytes = BM * BK * 2;            // 16 KiB
-constexpr int kBBytes = BN * BK * 2;            // 32 KiB
-constexpr int kStageBytes = kABytes + kBBytes;  // 48 KiB
 constexpr int kTmemCols = 512;
+constexpr int kTmemBufStride = 256;             // the two accumulators sit at columns 0 and 256
 constexpr int kThreads = 192;
-constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kMaxSmem = 232448;                // 227 KiB per CTA
+
+// Tile width BN (accumulator columns) is a template parameter: 256 by default, narrower tiles where they
+// remove a mostly empty last wave (e.g. N = 5120 over 148 SMs: 23 tiles of 224 fill 4.97 waves, 20 of 256 need 5 of 4.3).
+template <int BN>
+struct TileCfg {
+  static constexpr int kBBytes = BN * BK * 2;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kStagesFit = (kMaxSmem - 1024 - 256) / kStageBytes;
+  static constexpr int kStages = kStagesFit > 6 ? 6 : kStagesFit;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
 
 enum WaitTag { TAG_EMPTY = 1, TAG_FULL = 2, TAG_TMEM_EMPTY = 3, TAG_TMEM_FULL = 4 };
 
@@ -51,11 +59,14 @@ __device__ __forceinline__ void store_chunk_bf16(bf16 *dst, const float (&v)[32]
                        pack_bf16(v[8 * q + 4], v[8 * q + 5]), pack_bf16(v[8 * q + 6], v[8 * q + 7]));
 }
 
-template <int MODE>
+template <int MODE, int BN>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CUtensorMap tma_b, int m, int n,
                int k, bf16 *__restrict__ out, float *__restrict__ resid, DeviceStatus *status,
                const __grid_constant__ QkvRopeArgs qa) {
+  constexpr int kStages = TileCfg<BN>::kStages;
+  constexpr int kBBytes = TileCfg<BN>::kBBytes;
+  constexpr int kStageBytes = TileCfg<BN>::kStageBytes;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t *smem_gen = smem_raw + (smem_base - tc::smem_u32(smem_raw));
@@ -135,7 +146,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
         ok = tc::mbar_wait(tempty_bar(buf), acc_phase ^ 1, abort_flag, status, TAG_TMEM_EMPTY);
         if (!ok) break;
         tc::tc_fence_after();
-        const uint32_t d_tmem = tmem_base + buf * BN;
+        const uint32_t d_tmem = tmem_base + buf * kTmemBufStride;
         for (int kb = 0; kb < k_blocks; ++kb) {
           ok = tc::mbar_wait(full_bar(stage), phase, abort_flag, status, TAG_FULL);
           if (!ok) break;
@@ -167,7 +178,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
       if (!ok) break;
       tc::tc_fence_after();
       const int row = m0 + quarter * 32 + lane;
-      const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * BN;
+      const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * kTmemBufStride;
       if (MODE == GEMM_QKV_ROPE) {
         // columns of this tile are whole heads (head_dim divides 256); a head's pair (j, j + d/2) lies in
         // chunks c and c + d/64.  The row is token `row` of the call, at absolute position pos0 + row.
@@ -293,6 +304,41 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
   }
 }
 
+template <int MODE, int BN>
+int launch_gemm(const CUtensorMap &ta, const CUtensorMap &tb, int m, int n, int k, bf16 *out, float *resid,
+                DeviceStatus *status, const QkvRopeArgs &qa, int sms, cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    KV_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<MODE, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 TileCfg<BN>::kSmemBytes));
+    attr_set = true;
+  }
+  const int out_cols = (MODE == GEMM_SWIGLU) ? BN / 2 : BN;
+  const int tiles = ((m + BM - 1) / BM) * ((n + out_cols - 1) / out_cols);
+  const int grid = tiles < sms ? tiles : sms;
+  gemm_tc_kernel<MODE, BN><<<grid, kThreads, TileCfg<BN>::kSmemBytes, st>>>(ta, tb, m, n, k, out, resid, status, qa);
+  KV_COUNT_LAUNCH();
+  KV_CUDA(cudaGetLastError());
+  return KV_OK;
+}
+
+// Tile width that minimises (waves x tile width) for an M x N problem on `sms` SMs; ties go to the wider tile.
+int pick_bn(int m, int n, int sms) {
+  const int widths[5] = {256, 224, 192, 160, 128};
+  const long long m_tiles = (m + BM - 1) / BM;
+  int best = 256;
+  long long best_cost = -1;
+  for (int bn : widths) {
+    const long long tiles = m_tiles * ((n + bn - 1) / bn);
+    const long long cost = ((tiles + sms - 1) / sms) * bn;
+    if (best_cost < 0 || cost < best_cost) {
+      best_cost = cost;
+      best = bn;
+    }
+  }
+  return best;
+}
+
 }  // namespace
 
 int gemm_tc(const bf16 *a, int lda, const bf16 *w, int m, int n, int k, int mode, bf16 *out, float *resid,
@@ -308,38 +354,36 @@ int gemm_tc(const bf16 *a, int lda, const bf16 *w, int m, int n, int k, int mode
   }
   if ((k % 8) != 0 || (lda % 8) != 0 || (n % 8) != 0) return KV_ERR_SHAPE;
   if (((uintptr_t)a & 15) || ((uintptr_t)w & 15)) return KV_ERR_ARG;
-  CUtensorMap ta, tb;
-  int rc = tc::make_tmap_2d(&ta, a, m, k, lda, BM);
-  if (rc != KV_OK) return rc;
-  const long long w_rows = (mode == GEMM_SWIGLU) ? 2ll * n : n;
-  rc = tc::make_tmap_2d(&tb, w, w_rows, k, k, (mode == GEMM_SWIGLU) ? BN / 2 : BN);
-  if (rc != KV_OK) return rc;
-
   static int sms = 0;
   if (sms == 0) {
     int device = 0;
     KV_CUDA(cudaGetDevice(&device));
     KV_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
-    KV_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<GEMM_STORE_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-    KV_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<GEMM_RESID_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-    KV_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<GEMM_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-    KV_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<GEMM_QKV_ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
   }
-  const int out_cols = (mode == GEMM_SWIGLU) ? BN / 2 : BN;
-  const int tiles = ((m + BM - 1) / BM) * ((n + out_cols - 1) / out_cols);
-  const int grid = tiles < sms ? tiles : sms;
+  const int bn = (mode == GEMM_RESID_F32 || mode == GEMM_STORE_BF16) ? pick_bn(m, n, sms) : 256;
+  CUtensorMap ta, tb;
+  int rc = tc::make_tmap_2d(&ta, a, m, k, lda, BM);
+  if (rc != KV_OK) return rc;
+  const long long w_rows = (mode == GEMM_SWIGLU) ? 2ll * n : n;
+  rc = tc::make_tmap_2d(&tb, w, w_rows, k, k, (mode == GEMM_SWIGLU) ? bn / 2 : bn);
+  if (rc != KV_OK) return rc;
   DeviceStatus *status = reinterpret_cast<DeviceStatus *>(status_dev);
-  if (mode == GEMM_STORE_BF16)
-    gemm_tc_kernel<GEMM_STORE_BF16><<<grid, kThreads, kSmemBytes, st>>>(ta, tb, m, n, k, out, resid, status, qa);
-  else if (mode == GEMM_RESID_F32)
-    gemm_tc_kernel<GEMM_RESID_F32><<<grid, kThreads, kSmemBytes, st>>>(ta, tb, m, n, k, out, resid, status, qa);
-  else if (mode == GEMM_SWIGLU)
-    gemm_tc_kernel<GEMM_SWIGLU><<<grid, kThreads, kSmemBytes, st>>>(ta, tb, m, n, k, out, resid, status, qa);
-  else
-    gemm_tc_kernel<GEMM_QKV_ROPE><<<grid, kThreads, kSmemBytes, st>>>(ta, tb, m, n, k, out, resid, status, qa);
-  KV_COUNT_LAUNCH();
-  KV_CUDA(cudaGetLastError());
-  return KV_OK;
+#define KV_GEMM_CASE(MODE_, BN_) \
+  if (mode == MODE_ && bn == BN_) return launch_gemm<MODE_, BN_>(ta, tb, m, n, k, out, resid, status, qa, sms, st)
+  KV_GEMM_CASE(GEMM_RESID_F32, 256);
+  KV_GEMM_CASE(GEMM_RESID_F32, 224);
+  KV_GEMM_CASE(GEMM_RESID_F32, 192);
+  KV_GEMM_CASE(GEMM_RESID_F32, 160);
+  KV_GEMM_CASE(GEMM_RESID_F32, 128);
+  KV_GEMM_CASE(GEMM_STORE_BF16, 256);
+  KV_GEMM_CASE(GEMM_STORE_BF16, 224);
+  KV_GEMM_CASE(GEMM_STORE_BF16, 192);
+  KV_GEMM_CASE(GEMM_STORE_BF16, 160);
+  KV_GEMM_CASE(GEMM_STORE_BF16, 128);
+  KV_GEMM_CASE(GEMM_SWIGLU, 256);
+  KV_GEMM_CASE(GEMM_QKV_ROPE, 256);
+#undef KV_GEMM_CASE
+  return KV_ERR_ARG;
 }
 
 }  // namespace kvr

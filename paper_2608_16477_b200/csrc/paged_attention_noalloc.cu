@@ -48,8 +48,8 @@ extern "C" int32_t kv_op_paged_attention_noalloc(const float *q_dev, int32_t n_q
       cache == nullptr || cache->base_dev == nullptr)
     return KV_ERR_ARG;
   if (cache->num_blocks <= 0 || cache->block_size <= 0 || cache->n_kv_heads <= 0 || cache->elem_bytes != 2 ||
-      layer < 0 || layer >= cache->n_layers || n_q_heads % cache->n_kv_heads != 0 || cache->head_dim % 32 != 0 ||
-      cache->head_dim <= 0 || cache->head_dim > 256)
+      layer < 0 || layer >= cache->n_layers || n_q_heads % cache->n_kv_heads != 0 ||
+      (cache->head_dim != 64 && cache->head_dim != 128))
     return KV_ERR_SHAPE;
   // the fixed array bounds the context length: reject what does not fit instead of spilling past it
   if (paged_attention_scratch_bytes(n_q_heads, cache->head_dim, n_ctx) > kNoAllocScratchBytes) return KV_ERR_WORKSPACE;
