@@ -8,8 +8,9 @@
 //   warp 1      TMEM allocation and MMA issue:  S = Q K^T  (both operands K-major in shared memory),
 //               O += P V  (P read from TMEM, V as an MN-major shared-memory operand: no transposes).
 //   warps 4-7   softmax of tile a, warps 8-11 softmax of tile b: one thread per query row (= TMEM lane).
-//               Pass 1 reads the row of S for its maximum, pass 2 turns it into bf16 probabilities written
-//               back over the first half of S in TMEM.  Statistics stay in fp32; the running maximum is
+//               The row of S is read once into registers (setmaxnreg moves registers from warps 0-3 to the
+//               softmax warps), reduced to its maximum and turned into bf16 probabilities written back over
+//               the first half of S in TMEM.  Statistics stay in fp32; the running maximum is
 //               only advanced (and O rescaled in TMEM) when it grows by more than 8 in the log2 domain,
 //               which keeps exp2 arguments <= 8 and makes rescaling rare.
 // TMEM columns: S_a [0,128)  S_b [128,256)  O_a [256,256+D)  O_b [384,384+D).
@@ -27,6 +28,8 @@ constexpr int kKvStages = 2;
 constexpr int kAttnThreads = 384;   // 12 warps
 constexpr uint32_t kTmemS0 = 0, kTmemS1 = 128, kTmemO0 = 256, kTmemO1 = 384;
 constexpr float kRescaleThreshold = 8.0f;
+constexpr int kRegsOther = 72;      // registers per thread of warps 0-3 after the hand-back
+constexpr int kRegsSoftmax = 216;   // registers per thread of the softmax warps (128 x 72 + 256 x 216 <= 64 Ki)
 
 enum AttnTag { ATAG_Q = 11, ATAG_KV_EMPTY = 12, ATAG_K = 13, ATAG_V = 14, ATAG_S = 15, ATAG_P = 16, ATAG_O = 17 };
 
@@ -126,8 +129,11 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
   tc::tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
 
+  // the softmax warpgroups hold a full row of S in registers; warps 0-3 give registers back (first statement
+  // of every role so the register budget of each branch is known at compile time)
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
     if (lane == 0) {
       tc::tma_prefetch_desc(&tma_qkv);
       for (int t = 0; t < 2; ++t) {
@@ -152,6 +158,7 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
     if (lane == 0) {
       constexpr uint32_t idesc_qk = tc::umma_idesc_bf16(kBM, kBN);
       constexpr uint32_t idesc_pv = tc::umma_idesc_bf16(kBM, D) | (1u << 16);   // B (= V) is MN-major
@@ -200,8 +207,11 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
         }
       }
     }
-  } else if (warp >= 4) {
+  } else if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
+  } else {
     // ---------------------------------------------------------------- softmax warpgroups
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
     const int t = (warp - 4) >> 2;                 // 0: tile a, 1: tile b
     const int quarter = warp & 3;
     const int row_in_tile = quarter * 32 + lane;
@@ -218,17 +228,29 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
       tc::tc_fence_after();
       const bool diag = (j == n_kv - 1);
       const int limit = qi - j * kBN;              // keys with column > limit are masked
-      // pass 1: row maximum
+      // the whole row of S (128 fp32) in registers: four loads in flight, one wait
+      uint32_t r0[32], r1[32], r2[32], r3[32];
+      tc::tmem_ld32(s_t + 0, r0);
+      tc::tmem_ld32(s_t + 32, r1);
+      tc::tmem_ld32(s_t + 64, r2);
+      tc::tmem_ld32(s_t + 96, r3);
+      tc::tmem_ld_wait();
       float mx = -INFINITY;
-#pragma unroll 1
-      for (int c = 0; c < kBN / 32; ++c) {
-        uint32_t r[32];
-        tc::tmem_ld32(s_t + c * 32, r);
-        tc::tmem_ld_wait();
+      if (!diag) {
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
-          const float s = __uint_as_float(r[i]);
-          if (!diag || c * 32 + i <= limit) mx = fmaxf(mx, s);
+          mx = fmaxf(mx, fmaxf(fmaxf(__uint_as_float(r0[i]), __uint_as_float(r1[i])),
+                               fmaxf(__uint_as_float(r2[i]), __uint_as_float(r3[i]))));
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          if (i > limit) r0[i] = 0xff800000u;        // -inf
+          if (32 + i > limit) r1[i] = 0xff800000u;
+          if (64 + i > limit) r2[i] = 0xff800000u;
+          if (96 + i > limit) r3[i] = 0xff800000u;
+          mx = fmaxf(mx, fmaxf(fmaxf(__uint_as_float(r0[i]), __uint_as_float(r1[i])),
+                               fmaxf(__uint_as_float(r2[i]), __uint_as_float(r3[i]))));
         }
       }
       mx *= scale_log2;
@@ -254,26 +276,26 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
           tmem_st32(o_t + c * 32, r);
         }
       }
-      // pass 2: probabilities, written over S as packed bf16 (two keys per 32-bit column)
-#pragma unroll 1
-      for (int c = 0; c < kBN / 32; ++c) {
-        uint32_t r[32];
-        tc::tmem_ld32(s_t + c * 32, r);
-        tc::tmem_ld_wait();
+      // probabilities, written over S as packed bf16 (two keys per 32-bit column); masked scores are -inf -> 0
+      const float neg_m = -m_ref;
+      float sum0 = 0.f, sum1 = 0.f;
+      auto emit = [&](const uint32_t (&r)[32], int c) {
         uint32_t pk[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
-          float p0 = exp2f(__uint_as_float(r[2 * i]) * scale_log2 - m_ref);
-          float p1 = exp2f(__uint_as_float(r[2 * i + 1]) * scale_log2 - m_ref);
-          if (diag) {
-            if (c * 32 + 2 * i > limit) p0 = 0.f;
-            if (c * 32 + 2 * i + 1 > limit) p1 = 0.f;
-          }
-          l_sum += p0 + p1;
+          const float p0 = exp2f(fmaf(__uint_as_float(r[2 * i]), scale_log2, neg_m));
+          const float p1 = exp2f(fmaf(__uint_as_float(r[2 * i + 1]), scale_log2, neg_m));
+          sum0 += p0;
+          sum1 += p1;
           pk[i] = pack2(p0, p1);
         }
         tmem_st16(s_t + c * 16, pk);
-      }
+      };
+      emit(r0, 0);
+      emit(r1, 1);
+      emit(r2, 2);
+      emit(r3, 3);
+      l_sum += sum0 + sum1;
       tc::tmem_st_wait();
       tc::tc_fence_before();
       tc::mbar_arrive(bar(B_P, t));
