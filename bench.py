@@ -279,6 +279,39 @@ def run_ours(args):
             ms = float(t.item())
         return ms
 
+    # standalone pack / unpack bandwidth, rotating over disjoint block sets so every launch reads cold pages.
+    # Timed alone, before the compute-heavy steps pull the clocks down under the power cap: the same condition
+    # as the copy measurement the HBM peak comes from (the in-step times are in breakdown_ms_per_step).
+    n_sets = max(1, min(8, (pool_blocks - nb_total - 1) // max(nb_suffix, 1)))
+    sets_src = [perm_src[nb_total + 1 + i * nb_suffix: nb_total + 1 + (i + 1) * nb_suffix].copy() for i in range(n_sets)]
+    sets_dst = [perm_tgt[nb_total + 1 + i * nb_suffix: nb_total + 1 + (i + 1) * nb_suffix].copy() for i in range(n_sets)]
+    wires = [torch.empty(wire_elems, dtype=torch.int16, device="cuda") for _ in range(n_sets)]
+    payload = wire_elems * 2
+
+    def pack_all():
+        for i in range(n_sets):
+            kv.kv_pack_blocks(src, sets_src[i], wires[i])
+
+    def unpack_all():
+        for i in range(n_sets):
+            kv.kv_unpack_assemble(tgt, wires[i], logical, sets_dst[i], tgt_prefix, n, epoch=1, expected_epoch=1)
+    pack_all(); unpack_all()
+    torch.cuda.synchronize()
+
+    def graph_time(fn, reps=10):
+        """Device time per launch with the launches replayed from a CUDA graph, so that host-side call
+        overhead (longer than a ~45 us kernel) does not sit between consecutive launches."""
+        try:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                fn()
+            g.replay()
+            return timed(g.replay, reps) / (reps * n_sets), "cuda-graph replay"
+        except Exception:
+            return timed(fn, reps) / (reps * n_sets), "direct launches"
+    pack_ms, pack_how = graph_time(pack_all)
+    unpack_ms, _ = graph_time(unpack_all)
+
     for _ in range(max(args.warmup, 3)):
         step()
     kv.kv_check_device_status(ws_p)
@@ -302,25 +335,6 @@ def run_ours(args):
 
     step_e2e()
     e2e_ms = timed(step_e2e, args.steps)
-
-    # standalone pack / unpack bandwidth, rotating over disjoint block sets so every launch reads cold pages
-    n_sets = max(1, min(8, (pool_blocks - nb_total - 1) // max(nb_suffix, 1)))
-    sets_src = [perm_src[nb_total + 1 + i * nb_suffix: nb_total + 1 + (i + 1) * nb_suffix].copy() for i in range(n_sets)]
-    sets_dst = [perm_tgt[nb_total + 1 + i * nb_suffix: nb_total + 1 + (i + 1) * nb_suffix].copy() for i in range(n_sets)]
-    wires = [torch.empty(wire_elems, dtype=torch.int16, device="cuda") for _ in range(n_sets)]
-    payload = wire_elems * 2
-
-    def pack_all():
-        for i in range(n_sets):
-            kv.kv_pack_blocks(src, sets_src[i], wires[i])
-
-    def unpack_all():
-        for i in range(n_sets):
-            kv.kv_unpack_assemble(tgt, wires[i], logical, sets_dst[i], tgt_prefix, n, epoch=1, expected_epoch=1)
-    pack_all(); unpack_all()
-    reps = 5
-    pack_ms = timed(pack_all, reps) / (reps * n_sets)
-    unpack_ms = timed(unpack_all, reps) / (reps * n_sets)
 
     if rank != 0:
         if world > 1:
@@ -363,7 +377,8 @@ def run_ours(args):
                     "frac_of_bf16_burst_peak": flops / (prefill_ms * 1e-3) / 1e12 / pk["bf16_tflops"],
                     "frac_of_bf16_sustained_peak": flops / (prefill_ms * 1e-3) / 1e12 / pk["bf16_tflops_sustained"]},
         "pack": {"gbs": 2 * payload / (pack_ms * 1e-3) / 1e9, "frac_of_hbm": 2 * payload / (pack_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
-                 "us": pack_ms * 1e3, "payload_bytes": payload},
+                 "us": pack_ms * 1e3, "payload_bytes": payload,
+                 "timing": f"{pack_how} of {n_sets} launches over disjoint block sets"},
         "unpack": {"gbs": 2 * payload / (unpack_ms * 1e-3) / 1e9,
                    "frac_of_hbm": 2 * payload / (unpack_ms * 1e-3) / 1e9 / pk["hbm_gbs"], "us": unpack_ms * 1e3},
         "decode_step_ms": decode_ms,

@@ -122,6 +122,10 @@ int64_t kv_bytes_per_token(int32_t n_layers, int32_t n_kv_heads, int32_t head_di
  * prefill/decode call on it: KV_OK, or KV_ERR_DEVICE if a kernel's bounded wait ran out. */
 int32_t kv_check_device_status(const void *workspace_dev, void *stream);
 
+/* Synchronises `stream` and reports whether any pack/unpack kernel of this process gave up a bounded wait
+ * (KV_ERR_DEVICE; the copy it belonged to is then incomplete).  KV_OK otherwise. */
+int32_t kv_check_copy_status(void *stream);
+
 /* ---------------------------------------------------------------- the four operations */
 
 /* Target-side prefix reconstruction (Section 4.3 / Section 5: the target reconstructs the prefix KV

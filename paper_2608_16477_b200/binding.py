@@ -19,7 +19,7 @@ EXPORTS = [
     "kv_unpack_assemble", "kv_decode_step", "kv_pack_blocks_batched", "kv_unpack_blocks_batched",
     "kv_op_gemm", "kv_op_gemm_reference", "kv_op_rmsnorm",
     "kv_op_attention_prefill", "kv_paged_attention_scratch_bytes", "kv_op_paged_attention", "kv_fill_pattern",
-    "kv_profile_enable", "kv_profile_read", "kv_launch_count", "kv_op_paged_attention_noalloc",
+    "kv_profile_enable", "kv_profile_read", "kv_launch_count", "kv_op_paged_attention_noalloc", "kv_check_copy_status",
 ]
 
 PROFILE_KINDS = ("embed", "rmsnorm", "gemm_qkv", "rope_store", "attention", "gemm_o", "gemm_gate_up", "gemm_down",
@@ -95,6 +95,7 @@ def load(build_if_missing: bool = True):
         "kv_op_paged_attention": (i32, [vp, i32, C.POINTER(CacheDesc), i32, vp, i32, vp, i64, vp, vp]),
         "kv_fill_pattern": (i32, [vp, i64, C.c_uint64, i64, vp]),
         "kv_op_paged_attention_noalloc": (i32, [vp, i32, C.POINTER(CacheDesc), i32, vp, i32, vp, vp]),
+        "kv_check_copy_status": (i32, [vp]),
         "kv_profile_enable": (i32, [i32]),
         "kv_profile_read": (i32, [C.POINTER(C.c_float), C.POINTER(C.c_int64), i32]),
         "kv_launch_count": (i64, []),
@@ -364,3 +365,7 @@ def kv_op_paged_attention_noalloc(q, cache: PagedCache, layer, block_table_dev, 
     _check(load().kv_op_paged_attention_noalloc(_ptr(q), q.shape[0], C.byref(cache.desc), layer,
                                                 _ptr(block_table_dev), n_ctx, _ptr(out), _stream(stream)),
            "kv_op_paged_attention_noalloc")
+
+
+def kv_check_copy_status(stream=None) -> None:
+    _check(load().kv_check_copy_status(_stream(stream)), "kv_check_copy_status")

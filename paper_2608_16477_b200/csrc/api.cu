@@ -384,8 +384,8 @@ int32_t kv_prefill_prefix(kv_model *m, const kv_cache_desc *cache, const int32_t
   }
   if (logits_out_dev != nullptr) {
     ProfScope ps(PROF_LM_HEAD, st);
-    KV_TRY(rmsnorm_vec(w.x + (long long)(t - 1) * d.hidden, m->final_norm, d.hidden, d.rms_eps, w.xf, st));
-    KV_TRY(gemv(m->lm_head, w.xf, d.vocab, d.hidden, 0, logits_out_dev, st));
+    KV_TRY(gemv(m->lm_head, w.x + (long long)(t - 1) * d.hidden, d.vocab, d.hidden, 0, logits_out_dev, st,
+                m->final_norm, d.rms_eps));
   }
   return KV_OK;
 }
@@ -410,24 +410,19 @@ int32_t kv_decode_step(kv_model *m, const kv_cache_desc *cache, int32_t token_id
   if (workspace_bytes < w.bytes) return KV_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   const CacheView cv = make_view(cache);
-  const int qkv_dim = (d.n_q_heads + 2 * d.n_kv_heads) * d.head_dim;
   const int q_dim = d.n_q_heads * d.head_dim;
 
   KV_CUDA(cudaMemsetAsync(w.status, 0, sizeof(DeviceStatus), st));
   KV_CUDA(cudaMemcpyAsync(w.table, block_table_host, sizeof(int) * need_blocks, cudaMemcpyHostToDevice, st));
   { ProfScope ps(PROF_DECODE_OTHER, st); KV_TRY(embed_one(m->embed, token_id, d.hidden, w.x, st)); }
   for (int l = 0; l < d.n_layers; ++l) {
-    { ProfScope ps(PROF_DECODE_OTHER, st); KV_TRY(rmsnorm_vec(w.x, m->attn_norm[l], d.hidden, d.rms_eps, w.h, st)); }
-    { ProfScope ps(PROF_DECODE_GEMV, st); KV_TRY(gemv(m->w_qkv[l], w.h, qkv_dim, d.hidden, 0, w.qkv, st)); }
-    { ProfScope ps(PROF_DECODE_OTHER, st); KV_TRY(rope_store_kv_one(w.qkv, pos, d.n_q_heads, d.n_kv_heads, d.head_dim, d.rope_base, cv, l, w.table, st)); }
+    { ProfScope ps(PROF_DECODE_GEMV, st); KV_TRY(gemv_qkv_rope(m->w_qkv[l], w.x, m->attn_norm[l], d.rms_eps, d.hidden, pos, d.n_q_heads, d.n_kv_heads, d.head_dim, d.rope_base, cv, l, w.table, w.qkv, st)); }
     { ProfScope ps(PROF_DECODE_ATTENTION, st); KV_TRY(paged_attention(w.qkv, d.n_q_heads, cv, l, w.table, n_ctx, w.scratch, w.o, st)); }
     { ProfScope ps(PROF_DECODE_GEMV, st); KV_TRY(gemv(m->w_o[l], w.o, d.hidden, q_dim, 1, w.x, st)); }
-    { ProfScope ps(PROF_DECODE_OTHER, st); KV_TRY(rmsnorm_vec(w.x, m->ffn_norm[l], d.hidden, d.rms_eps, w.h, st)); }
-    { ProfScope ps(PROF_DECODE_GEMV, st); KV_TRY(gemv(m->w_gate_up[l], w.h, d.ffn, d.hidden, 2, w.mid, st)); }
+    { ProfScope ps(PROF_DECODE_GEMV, st); KV_TRY(gemv(m->w_gate_up[l], w.x, d.ffn, d.hidden, 2, w.mid, st, m->ffn_norm[l], d.rms_eps)); }
     { ProfScope ps(PROF_DECODE_GEMV, st); KV_TRY(gemv(m->w_down[l], w.mid, d.hidden, d.ffn, 1, w.x, st)); }
   }
-  { ProfScope ps(PROF_DECODE_OTHER, st); KV_TRY(rmsnorm_vec(w.x, m->final_norm, d.hidden, d.rms_eps, w.h, st)); }
-  { ProfScope ps(PROF_LM_HEAD, st); KV_TRY(gemv(m->lm_head, w.h, d.vocab, d.hidden, 0, logits_out_dev, st)); }
+  { ProfScope ps(PROF_LM_HEAD, st); KV_TRY(gemv(m->lm_head, w.x, d.vocab, d.hidden, 0, logits_out_dev, st, m->final_norm, d.rms_eps)); }
   return KV_OK;
 }
 
@@ -585,6 +580,8 @@ int32_t kv_op_paged_attention(const float *q_dev, int32_t n_q_heads, const kv_ca
   return paged_attention(q_dev, n_q_heads, make_view(cache), layer, block_table_dev, n_ctx, scratch_dev, out_dev,
                          (cudaStream_t)stream);
 }
+
+int32_t kv_check_copy_status(void *stream) { return copy_wait_expired((cudaStream_t)stream); }
 
 int32_t kv_profile_enable(int32_t on) {
   g_prof_on = on != 0;

@@ -86,11 +86,14 @@ int attention_prefill(const bf16 *qkv, int n_tokens, int pos0, int n_q_heads, in
 
 // decode-step kernels (one token, fp32 activations)
 int embed_one(const bf16 *embed, int token, int hidden, float *x, cudaStream_t st);
-int rmsnorm_vec(const float *x, const bf16 *gain, int dim, float eps, float *out, cudaStream_t st);
 // y[n] (+)= sum_k W[n,k] x[k]; mode 0 store, 1 add into y, 2 swiglu over (gate | up) rows
-int gemv(const bf16 *w, const float *x, int n, int k, int mode, float *y, cudaStream_t st);
-int rope_store_kv_one(float *qkv, int pos, int n_q_heads, int n_kv_heads, int head_dim, float base,
-                      CacheView cache, int layer, const int *block_table_dev, cudaStream_t st);
+// gain != nullptr fuses RMSNorm(x, gain, eps) into the product (modes 0 and 2)
+int gemv(const bf16 *w, const float *x, int n, int k, int mode, float *y, cudaStream_t st,
+         const bf16 *gain = nullptr, float eps = 0.f);
+// RMSNorm + QKV projection + RoPE + K/V append of one decode token; q_out = rotated fp32 queries
+int gemv_qkv_rope(const bf16 *w_qkv, const float *x, const bf16 *gain, float eps, int hidden, int pos, int n_q_heads,
+                  int n_kv_heads, int head_dim, float base, CacheView cache, int layer, const int *block_table_dev,
+                  float *q_out, cudaStream_t st);
 long long paged_attention_scratch_bytes(int n_q_heads, int head_dim, int n_ctx);
 int paged_attention(const float *q, int n_q_heads, CacheView cache, int layer, const int *block_table_dev,
                     int n_ctx, void *scratch, float *out, cudaStream_t st);
@@ -98,6 +101,7 @@ int paged_attention(const float *q, int n_q_heads, CacheView cache, int layer, c
 int copy_pages(CacheView cache, int n_layers, const int *ids_host, int n_blocks, char *wire,
                int wire_layout, int total_blocks_in_wire, int first_block_in_wire, bool to_wire,
                cudaStream_t st);
+int copy_wait_expired(cudaStream_t st);   // KV_ERR_DEVICE if a pack/unpack kernel gave up a wait
 int fill_pattern(void *dst, long long bytes, unsigned long long seed, long long offset, cudaStream_t st);
 
 }  // namespace kvr

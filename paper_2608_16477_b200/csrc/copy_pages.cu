@@ -2,16 +2,26 @@
 //
 // One launch moves every page of up to kMaxIds logical blocks: block ids travel in the kernel
 // parameter block, so no device-side staging of the id list and no extra copy precede the kernel.
-// A page (block_size * n_kv_heads * head_dim bf16) is contiguous on both sides; each CTA streams
-// 16 KiB pieces of pages with 16-byte vector loads/stores, four independent loads in flight per
-// thread.  HBM-bound: 2 * page bytes of traffic per page, nothing is re-read.
+// A page (block_size * n_kv_heads * head_dim bf16) is contiguous on both sides; it moves as 16 KiB
+// bulk copies (cp.async.bulk) through a shared-memory ring.  HBM-bound: 2 * page bytes of traffic
+// per page, nothing is re-read.
 #include "common.cuh"
 
 namespace kvr {
 
 constexpr int kMaxIds = 960;          // keeps the parameter block under 4 KiB
-constexpr int kCopyThreads = 256;
-constexpr int kUnroll = 4;            // 16-byte vectors per thread per piece
+#ifndef KV_COPY_PIECE
+#define KV_COPY_PIECE 16384
+#define KV_COPY_BUFS 8
+#define KV_COPY_LAG 4
+#define KV_COPY_CTAS 1
+#endif
+constexpr int kPieceBytes = KV_COPY_PIECE;   // bytes per bulk copy
+constexpr int kBufs = KV_COPY_BUFS;          // shared-memory ring: 128 KiB per CTA, one CTA per SM (measured best: ~128 KiB in flight per SM)
+constexpr int kLag = KV_COPY_LAG;            // stores left in flight before a slot is refilled (kBufs - kLag loads in flight)
+constexpr int kCopyThreads = 32;
+constexpr int kCtasPerSm = KV_COPY_CTAS;
+constexpr long long kCopyWaitLimit = 2000000000ll;   // cycles (~1 s): far beyond any legitimate wait
 
 struct PageCopyParams {
   CacheView cache;
@@ -21,17 +31,54 @@ struct PageCopyParams {
   int layout;                // KV_WIRE_BLOCK_MAJOR / KV_WIRE_LAYER_MAJOR
   int total_blocks;          // blocks in the whole wire buffer (layer-major stride)
   int first_block;           // index of this launch's first block inside the wire buffer
-  int vec_per_page;          // page bytes / 16
-  int pieces_per_page;       // ceil(vec_per_page / (kCopyThreads * kUnroll))
+  int page_bytes;
+  int pieces_per_page;       // ceil(page_bytes / kPieceBytes)
   int ids[kMaxIds];
 };
 
+// Set by a copy kernel whose bounded wait ran out (the kernel then stops copying and returns).
+__device__ int g_copy_wait_expired = 0;
+
+__device__ __forceinline__ uint32_t cp_smem(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ bool cp_wait(uint32_t bar, uint32_t parity) {
+  const long long t0 = clock64();
+  for (uint32_t it = 0;; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    if (ok) return true;
+    if ((it & 0xff) == 0xff && clock64() - t0 > kCopyWaitLimit) {
+      g_copy_wait_expired = 1;
+      return false;
+    }
+  }
+}
+
+// One thread per CTA drives a ring of bulk copies: global -> shared (completion on an mbarrier), then
+// shared -> global (bulk group).  Neither the LSU nor registers touch the payload, so the achieved
+// bandwidth does not depend on the SM clock.  A slot is refilled once the store that read it has
+// finished reading (wait_group.read), which keeps kBufs - kLag loads and kLag stores in flight per CTA.
 template <bool TO_WIRE>
 __global__ void __launch_bounds__(kCopyThreads) copy_pages_kernel(const __grid_constant__ PageCopyParams p) {
-  const long long page_bytes = (long long)p.vec_per_page * 16;
+  extern __shared__ __align__(128) unsigned char ring[];
+  __shared__ __align__(8) unsigned long long full[kBufs];
+  if (threadIdx.x != 0) return;
   const long long n_pages = (long long)p.n_blocks * p.n_layers * 2;
   const long long n_items = n_pages * p.pieces_per_page;
-  for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
+  // this CTA's items: blockIdx.x, blockIdx.x + gridDim.x, ...
+  const long long mine = (n_items - blockIdx.x + gridDim.x - 1) / gridDim.x;
+  if (mine <= 0) return;
+  for (int b = 0; b < kBufs; ++b)
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(cp_smem(&full[b])));
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+
+  auto locate = [&](long long k, const char *&src, char *&dst, uint32_t &bytes) {
+    const long long item = blockIdx.x + k * gridDim.x;
     const long long pg = item / p.pieces_per_page;
     const int piece = (int)(item - pg * p.pieces_per_page);
     const int i = (int)(pg / (2 * p.n_layers));
@@ -42,30 +89,56 @@ __global__ void __launch_bounds__(kCopyThreads) copy_pages_kernel(const __grid_c
       wire_page = ((long long)(p.first_block + i) * p.n_layers + layer) * 2 + kv;
     else
       wire_page = ((long long)layer * 2 + kv) * p.total_blocks + p.first_block + i;
-    int4 *cpage = reinterpret_cast<int4 *>(p.cache.page(layer, kv, p.ids[i]));
-    int4 *wpage = reinterpret_cast<int4 *>(p.wire + wire_page * page_bytes);
-    const int4 *src = TO_WIRE ? cpage : wpage;
-    int4 *dst = TO_WIRE ? wpage : cpage;
-    const int v0 = piece * kCopyThreads * kUnroll + threadIdx.x;
-    int4 r[kUnroll];
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      const int v = v0 + u * kCopyThreads;
-      if (v < p.vec_per_page) r[u] = __ldcs(src + v);
-    }
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      const int v = v0 + u * kCopyThreads;
-      if (v < p.vec_per_page) __stcs(dst + v, r[u]);
+    const long long off = (long long)piece * kPieceBytes;
+    char *c = p.cache.page(layer, kv, p.ids[i]) + off;
+    char *w = p.wire + wire_page * p.page_bytes + off;
+    src = TO_WIRE ? c : w;
+    dst = TO_WIRE ? w : c;
+    const long long left = p.page_bytes - off;
+    bytes = (uint32_t)(left < kPieceBytes ? left : kPieceBytes);
+  };
+  auto load = [&](long long k) {
+    const int slot = (int)(k % kBufs);
+    const char *src; char *dst; uint32_t bytes;
+    locate(k, src, dst, bytes);
+    const uint32_t bar = cp_smem(&full[slot]);
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(cp_smem(ring + slot * kPieceBytes)), "l"(src), "r"(bytes), "r"(bar) : "memory");
+  };
+
+  const long long prologue = mine < kBufs ? mine : kBufs;
+  for (long long k = 0; k < prologue; ++k) load(k);
+  for (long long k = 0; k < mine; ++k) {
+    const int slot = (int)(k % kBufs);
+    if (!cp_wait(cp_smem(&full[slot]), (uint32_t)((k / kBufs) & 1))) break;
+    const char *src; char *dst; uint32_t bytes;
+    locate(k, src, dst, bytes);
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 ::"l"(dst), "r"(cp_smem(ring + slot * kPieceBytes)), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    // refill the slot of item k - kLag once its store has read it: up to kLag younger stores stay pending, so
+    // the issuing thread never waits on the store it has just issued
+    if (k >= kLag && k - kLag + kBufs < mine) {
+      asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kLag) : "memory");
+      load(k - kLag + kBufs);
     }
   }
+  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // all stores complete before the CTA exits
 }
 
 int copy_pages(CacheView cache, int n_layers, const int *ids_host, int n_blocks, char *wire, int wire_layout,
                int total_blocks_in_wire, int first_block_in_wire, bool to_wire, cudaStream_t st) {
-  int device = 0, sms = 148;
-  KV_CUDA(cudaGetDevice(&device));
-  KV_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+  static int sms = 0;
+  if (sms == 0) {
+    int device = 0;
+    KV_CUDA(cudaGetDevice(&device));
+    KV_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+    KV_CUDA(cudaFuncSetAttribute(copy_pages_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kBufs * kPieceBytes));
+    KV_CUDA(cudaFuncSetAttribute(copy_pages_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kBufs * kPieceBytes));
+  }
   for (int done = 0; done < n_blocks; done += kMaxIds) {
     PageCopyParams p;
     p.cache = cache;
@@ -75,20 +148,27 @@ int copy_pages(CacheView cache, int n_layers, const int *ids_host, int n_blocks,
     p.layout = wire_layout;
     p.total_blocks = total_blocks_in_wire;
     p.first_block = first_block_in_wire + done;
-    p.vec_per_page = (int)(cache.page_bytes() / 16);
-    p.pieces_per_page = (p.vec_per_page + kCopyThreads * kUnroll - 1) / (kCopyThreads * kUnroll);
+    p.page_bytes = (int)cache.page_bytes();
+    p.pieces_per_page = (p.page_bytes + kPieceBytes - 1) / kPieceBytes;
     for (int i = 0; i < p.n_blocks; ++i) p.ids[i] = ids_host[done + i];
     const long long items = (long long)p.n_blocks * n_layers * 2 * p.pieces_per_page;
-    const long long cap = (long long)sms * 8;   // 8 resident CTAs of 256 threads per SM
+    const long long cap = (long long)sms * kCtasPerSm;
     const int grid = (int)(items < cap ? items : cap);
     if (to_wire)
-      copy_pages_kernel<true><<<grid, kCopyThreads, 0, st>>>(p);
+      copy_pages_kernel<true><<<grid, kCopyThreads, kBufs * kPieceBytes, st>>>(p);
     else
-      copy_pages_kernel<false><<<grid, kCopyThreads, 0, st>>>(p);
+      copy_pages_kernel<false><<<grid, kCopyThreads, kBufs * kPieceBytes, st>>>(p);
     KV_COUNT_LAUNCH();
   KV_CUDA(cudaGetLastError());
   }
   return KV_OK;
+}
+
+int copy_wait_expired(cudaStream_t st) {
+  int flag = 0;
+  KV_CUDA(cudaStreamSynchronize(st));
+  KV_CUDA(cudaMemcpyFromSymbol(&flag, g_copy_wait_expired, sizeof(int)));
+  return flag ? KV_ERR_DEVICE : KV_OK;
 }
 
 // Counter-based fill: word w = mix(seed + w); the host-side generator computes the same function.

@@ -3,6 +3,8 @@
 // table with the keys split across CTAs (flash-decoding) and a second pass merging the splits.
 #include <float.h>
 
+#include <cstring>
+
 #include "common.cuh"
 
 namespace kvr {
@@ -26,28 +28,6 @@ int embed_one(const bf16 *embed, int token, int hidden, float *x, cudaStream_t s
   return KV_OK;
 }
 
-__global__ void __launch_bounds__(1024) rmsnorm_vec_kernel(const float *__restrict__ x,
-                                                           const bf16 *__restrict__ gain, int dim, float eps,
-                                                           float *__restrict__ out) {
-  __shared__ float red[32];
-  float ss = 0.f;
-  for (int c = threadIdx.x; c < dim; c += blockDim.x) ss += x[c] * x[c];
-  ss = warp_sum_d(ss);
-  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
-  __syncthreads();
-  float t = (threadIdx.x & 31) < (blockDim.x >> 5) ? red[threadIdx.x & 31] : 0.f;
-  t = warp_sum_d(t);
-  const float inv = rsqrtf(t / (float)dim + eps);
-  for (int c = threadIdx.x; c < dim; c += blockDim.x) out[c] = x[c] * inv * __bfloat162float(gain[c]);
-}
-
-int rmsnorm_vec(const float *x, const bf16 *gain, int dim, float eps, float *out, cudaStream_t st) {
-  rmsnorm_vec_kernel<<<1, 1024, 0, st>>>(x, gain, dim, eps, out);
-  KV_COUNT_LAUNCH();
-  KV_CUDA(cudaGetLastError());
-  return KV_OK;
-}
-
 __device__ __forceinline__ float dot8(uint4 wraw, float4 x0, float4 x1) {
   const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&wraw);
   float2 a = __bfloat1622float2(h[0]), b = __bfloat1622float2(h[1]);
@@ -55,99 +35,171 @@ __device__ __forceinline__ float dot8(uint4 wraw, float4 x0, float4 x1) {
   return a.x * x0.x + a.y * x0.y + b.x * x0.z + b.y * x0.w + c.x * x1.x + c.y * x1.y + d.x * x1.z + d.y * x1.w;
 }
 
-// Warp per output row; W row-major [rows, k] bf16 streamed once, x fp32 (L1/L2 resident).
-// MODE 0: y[n] = W[n].x   MODE 1: y[n] += W[n].x   MODE 2: y[n] = silu(W[n].x) * (W[n + N].x)
+// Matrix-vector products of the decode step.  A warp streams TWO weight rows (bf16, 16-byte loads, four
+// vectors of each row in flight per lane) against the fp32 activation vector, which stays in L1/L2.
+// NORM fuses the preceding RMSNorm: the warp accumulates sum(x^2) from the values it loads anyway and
+// computes W . (x * gain) * rsqrt(mean(x^2) + eps), so no separate normalisation launch is needed.
+// Epilogues: STORE rows (2u, 2u+1); ADD into the residual; SWIGLU rows (u, u + n) -> silu(a) * b;
+// QKV rows (j, j + d/2) of one head -> RoPE rotation, q to the fp32 query vector, k and v (bf16) appended
+// to the paged cache.
+enum GemvEpi { GEMV_STORE = 0, GEMV_ADD = 1, GEMV_SWIGLU = 2, GEMV_QKV = 3 };
 constexpr int kGemvWarps = 8;
-template <int MODE>
-__global__ void __launch_bounds__(kGemvWarps * 32) gemv_kernel(const bf16 *__restrict__ w,
-                                                               const float *__restrict__ x, int n, int k,
-                                                               float *__restrict__ y) {
+
+struct GemvQkvArgs {
+  CacheView cache;
+  const int *block_table;
+  int pos, layer, head_dim, n_q_heads, n_kv_heads;
+  float base;
+};
+
+template <int EPI, bool NORM>
+__global__ void __launch_bounds__(kGemvWarps * 32) gemv2_kernel(const bf16 *__restrict__ w,
+                                                                const float *__restrict__ x,
+                                                                const bf16 *__restrict__ gain, float eps, int n,
+                                                                int k, float *__restrict__ y,
+                                                                const __grid_constant__ GemvQkvArgs qa) {
   const int lane = threadIdx.x & 31;
-  const int row = blockIdx.x * kGemvWarps + (threadIdx.x >> 5);
-  if (row >= n) return;
-  const int nvec = k / 8;
-  const uint4 *wr = reinterpret_cast<const uint4 *>(w + (long long)row * k);
-  const uint4 *wr2 = reinterpret_cast<const uint4 *>(w + (long long)(row + n) * k);
-  const float4 *xv = reinterpret_cast<const float4 *>(x);
-  float acc = 0.f, acc2 = 0.f;
-  int v = lane;
-  for (; v + 96 < nvec; v += 128) {
-    uint4 w0 = __ldcs(wr + v), w1 = __ldcs(wr + v + 32), w2 = __ldcs(wr + v + 64), w3 = __ldcs(wr + v + 96);
-    uint4 u0, u1, u2, u3;
-    if (MODE == 2) { u0 = __ldcs(wr2 + v); u1 = __ldcs(wr2 + v + 32); u2 = __ldcs(wr2 + v + 64); u3 = __ldcs(wr2 + v + 96); }
-    float4 a0 = xv[2 * v], a1 = xv[2 * v + 1], b0 = xv[2 * (v + 32)], b1 = xv[2 * (v + 32) + 1];
-    float4 c0 = xv[2 * (v + 64)], c1 = xv[2 * (v + 64) + 1], d0 = xv[2 * (v + 96)], d1 = xv[2 * (v + 96) + 1];
-    acc += dot8(w0, a0, a1) + dot8(w1, b0, b1) + dot8(w2, c0, c1) + dot8(w3, d0, d1);
-    if (MODE == 2) acc2 += dot8(u0, a0, a1) + dot8(u1, b0, b1) + dot8(u2, c0, c1) + dot8(u3, d0, d1);
-  }
-  for (; v < nvec; v += 32) {
-    float4 a0 = xv[2 * v], a1 = xv[2 * v + 1];
-    acc += dot8(__ldcs(wr + v), a0, a1);
-    if (MODE == 2) acc2 += dot8(__ldcs(wr2 + v), a0, a1);
-  }
-  acc = warp_sum_d(acc);
-  if (MODE == 2) acc2 = warp_sum_d(acc2);
-  if (lane == 0) {
-    if (MODE == 0) y[row] = acc;
-    if (MODE == 1) y[row] += acc;
-    if (MODE == 2) y[row] = acc / (1.f + __expf(-acc)) * acc2;
-  }
-}
-
-int gemv(const bf16 *w, const float *x, int n, int k, int mode, float *y, cudaStream_t st) {
-  const int grid = (n + kGemvWarps - 1) / kGemvWarps;
-  if (mode == 0) gemv_kernel<0><<<grid, kGemvWarps * 32, 0, st>>>(w, x, n, k, y);
-  else if (mode == 1) gemv_kernel<1><<<grid, kGemvWarps * 32, 0, st>>>(w, x, n, k, y);
-  else gemv_kernel<2><<<grid, kGemvWarps * 32, 0, st>>>(w, x, n, k, y);
-  KV_COUNT_LAUNCH();
-  KV_CUDA(cudaGetLastError());
-  return KV_OK;
-}
-
-// Rotate the Q and K heads of the fp32 qkv vector in place and append K/V (bf16) to the cache.
-// The d/2 angles pos * base^(-2j/d) are formed once in fp64 (one thread per frequency) and shared.
-__global__ void __launch_bounds__(256) rope_store_kv_one_kernel(float *__restrict__ qkv, int pos, int n_q_heads,
-                                                                int n_kv_heads, int head_dim, float base,
-                                                                CacheView cache, int layer,
-                                                                const int *__restrict__ block_table) {
-  __shared__ float2 cs[128];
-  const int half = head_dim / 2;
-  for (int j = threadIdx.x; j < half; j += blockDim.x) {
-    double s, c;
-    sincos((double)pos * pow((double)base, -(double)j / (double)half), &s, &c);
-    cs[j] = make_float2((float)c, (float)s);
-  }
-  __syncthreads();
-  const int block = block_table[pos / cache.block_size];
-  const int slot = pos % cache.block_size;
-  bf16 *kpage = reinterpret_cast<bf16 *>(cache.page(layer, 0, block)) + (long long)slot * n_kv_heads * head_dim;
-  bf16 *vpage = reinterpret_cast<bf16 *>(cache.page(layer, 1, block)) + (long long)slot * n_kv_heads * head_dim;
-  const int n_rot = (n_q_heads + n_kv_heads) * half;
-  for (int idx = threadIdx.x; idx < n_rot; idx += blockDim.x) {
-    const int head = idx / half, j = idx - head * half;
-    const float2 c = cs[j];
-    float *h = qkv + head * head_dim;
-    const float a = h[j], b = h[j + half];
-    const float ra = a * c.x - b * c.y, rb = b * c.x + a * c.y;
-    h[j] = ra;
-    h[j + half] = rb;
-    if (head >= n_q_heads) {
-      bf16 *kd = kpage + (head - n_q_heads) * head_dim;
-      kd[j] = __float2bfloat16_rn(ra);
-      kd[j + half] = __float2bfloat16_rn(rb);
+  const int unit = blockIdx.x * kGemvWarps + (threadIdx.x >> 5);
+  int row_a, row_b;
+  bool has_b = true;
+  if (EPI == GEMV_SWIGLU) {
+    if (unit >= n) return;
+    row_a = unit;
+    row_b = unit + n;
+  } else if (EPI == GEMV_QKV) {
+    const int half = qa.head_dim >> 1;
+    if (unit >= n / 2) return;
+    const int head = unit / half, j = unit - head * half;
+    row_a = head * qa.head_dim + j;
+    row_b = row_a + half;
+  } else {
+    if (2 * unit >= n) return;
+    row_a = 2 * unit;
+    row_b = row_a + 1;
+    if (row_b >= n) {
+      row_b = row_a;
+      has_b = false;
     }
   }
-  const float *v = qkv + (n_q_heads + n_kv_heads) * head_dim;
-  for (int c = threadIdx.x; c < n_kv_heads * head_dim; c += blockDim.x) vpage[c] = __float2bfloat16_rn(v[c]);
+  const int nvec = k / 8;
+  const uint4 *wa = reinterpret_cast<const uint4 *>(w + (long long)row_a * k);
+  const uint4 *wb = reinterpret_cast<const uint4 *>(w + (long long)row_b * k);
+  const float4 *xv = reinterpret_cast<const float4 *>(x);
+  const uint4 *gv = reinterpret_cast<const uint4 *>(gain);
+  float acc_a = 0.f, acc_b = 0.f, ss = 0.f;
+  auto step = [&](uint4 ra, uint4 rb, int v) {
+    float4 x0 = xv[2 * v], x1 = xv[2 * v + 1];
+    if (NORM) {
+      ss += x0.x * x0.x + x0.y * x0.y + x0.z * x0.z + x0.w * x0.w + x1.x * x1.x + x1.y * x1.y + x1.z * x1.z +
+            x1.w * x1.w;
+      const uint4 graw = gv[v];
+      const __nv_bfloat162 *gh = reinterpret_cast<const __nv_bfloat162 *>(&graw);
+      const float2 g0 = __bfloat1622float2(gh[0]), g1 = __bfloat1622float2(gh[1]);
+      const float2 g2 = __bfloat1622float2(gh[2]), g3 = __bfloat1622float2(gh[3]);
+      x0.x *= g0.x; x0.y *= g0.y; x0.z *= g1.x; x0.w *= g1.y;
+      x1.x *= g2.x; x1.y *= g2.y; x1.z *= g3.x; x1.w *= g3.y;
+    }
+    acc_a += dot8(ra, x0, x1);
+    acc_b += dot8(rb, x0, x1);
+  };
+  int v = lane;
+  for (; v + 96 < nvec; v += 128) {
+    const uint4 a0 = __ldcs(wa + v), a1 = __ldcs(wa + v + 32), a2 = __ldcs(wa + v + 64), a3 = __ldcs(wa + v + 96);
+    const uint4 b0 = __ldcs(wb + v), b1 = __ldcs(wb + v + 32), b2 = __ldcs(wb + v + 64), b3 = __ldcs(wb + v + 96);
+    step(a0, b0, v);
+    step(a1, b1, v + 32);
+    step(a2, b2, v + 64);
+    step(a3, b3, v + 96);
+  }
+  for (; v < nvec; v += 32) step(__ldcs(wa + v), __ldcs(wb + v), v);
+  acc_a = warp_sum_d(acc_a);
+  acc_b = warp_sum_d(acc_b);
+  if (NORM) {
+    ss = warp_sum_d(ss);
+    const float inv = rsqrtf(ss / (float)k + eps);
+    acc_a *= inv;
+    acc_b *= inv;
+  }
+  if (lane != 0) return;
+  if (EPI == GEMV_STORE) {
+    y[row_a] = acc_a;
+    if (has_b) y[row_b] = acc_b;
+  } else if (EPI == GEMV_ADD) {
+    y[row_a] += acc_a;
+    if (has_b) y[row_b] += acc_b;
+  } else if (EPI == GEMV_SWIGLU) {
+    y[row_a] = acc_a / (1.f + __expf(-acc_a)) * acc_b;
+  } else {
+    const int d = qa.head_dim, half = d >> 1;
+    const int head = row_a / d, j = row_a - head * d;
+    const int block = qa.block_table[qa.pos / qa.cache.block_size];
+    const long long slot_off = (long long)(qa.pos % qa.cache.block_size) * qa.n_kv_heads * d;
+    if (head < qa.n_q_heads + qa.n_kv_heads) {
+      double sn, cs;
+      sincos((double)qa.pos * pow((double)qa.base, -(double)j / (double)half), &sn, &cs);
+      const float ra = acc_a * (float)cs - acc_b * (float)sn;
+      const float rb = acc_b * (float)cs + acc_a * (float)sn;
+      if (head < qa.n_q_heads) {
+        y[row_a] = ra;
+        y[row_b] = rb;
+      } else {
+        bf16 *kp = reinterpret_cast<bf16 *>(qa.cache.page(qa.layer, 0, block)) + slot_off + (head - qa.n_q_heads) * d;
+        kp[j] = __float2bfloat16_rn(ra);
+        kp[j + half] = __float2bfloat16_rn(rb);
+      }
+    } else {
+      bf16 *vp = reinterpret_cast<bf16 *>(qa.cache.page(qa.layer, 1, block)) + slot_off +
+                 (head - qa.n_q_heads - qa.n_kv_heads) * d;
+      vp[j] = __float2bfloat16_rn(acc_a);
+      vp[j + half] = __float2bfloat16_rn(acc_b);
+    }
+  }
 }
 
-int rope_store_kv_one(float *qkv, int pos, int n_q_heads, int n_kv_heads, int head_dim, float base,
-                      CacheView cache, int layer, const int *block_table_dev, cudaStream_t st) {
-  rope_store_kv_one_kernel<<<1, 256, 0, st>>>(qkv, pos, n_q_heads, n_kv_heads, head_dim, base, cache, layer,
-                                              block_table_dev);
+template <int EPI, bool NORM>
+static int launch_gemv2(const bf16 *w, const float *x, const bf16 *gain, float eps, int n, int k, float *y,
+                        const GemvQkvArgs &qa, cudaStream_t st) {
+  const int units = (EPI == GEMV_SWIGLU) ? n : (n + 1) / 2;
+  const int grid = (units + kGemvWarps - 1) / kGemvWarps;
+  gemv2_kernel<EPI, NORM><<<grid, kGemvWarps * 32, 0, st>>>(w, x, gain, eps, n, k, y, qa);
   KV_COUNT_LAUNCH();
   KV_CUDA(cudaGetLastError());
   return KV_OK;
+}
+
+// mode 0 store, 1 add into y, 2 swiglu over (gate | up) rows.  gain != nullptr fuses RMSNorm(x, gain, eps).
+int gemv(const bf16 *w, const float *x, int n, int k, int mode, float *y, cudaStream_t st, const bf16 *gain,
+         float eps) {
+  GemvQkvArgs qa;
+  memset(&qa, 0, sizeof(qa));
+  if (k % 8 != 0) return KV_ERR_SHAPE;
+  if (gain != nullptr) {
+    if (mode == 0) return launch_gemv2<GEMV_STORE, true>(w, x, gain, eps, n, k, y, qa, st);
+    if (mode == 2) return launch_gemv2<GEMV_SWIGLU, true>(w, x, gain, eps, n, k, y, qa, st);
+    return KV_ERR_ARG;
+  }
+  if (mode == 0) return launch_gemv2<GEMV_STORE, false>(w, x, nullptr, 0.f, n, k, y, qa, st);
+  if (mode == 1) return launch_gemv2<GEMV_ADD, false>(w, x, nullptr, 0.f, n, k, y, qa, st);
+  return launch_gemv2<GEMV_SWIGLU, false>(w, x, nullptr, 0.f, n, k, y, qa, st);
+}
+
+// Fused decode-step front end of a layer: RMSNorm + QKV projection + RoPE + K/V append.
+// q_out receives the rotated fp32 query vector [n_q_heads * head_dim].
+int gemv_qkv_rope(const bf16 *w_qkv, const float *x, const bf16 *gain, float eps, int hidden, int pos, int n_q_heads,
+                  int n_kv_heads, int head_dim, float base, CacheView cache, int layer, const int *block_table_dev,
+                  float *q_out, cudaStream_t st) {
+  GemvQkvArgs qa;
+  qa.cache = cache;
+  qa.block_table = block_table_dev;
+  qa.pos = pos;
+  qa.layer = layer;
+  qa.head_dim = head_dim;
+  qa.n_q_heads = n_q_heads;
+  qa.n_kv_heads = n_kv_heads;
+  qa.base = base;
+  if (hidden % 8 != 0) return KV_ERR_SHAPE;
+  const int n = (n_q_heads + 2 * n_kv_heads) * head_dim;
+  return launch_gemv2<GEMV_QKV, true>(w_qkv, x, gain, eps, n, hidden, q_out, qa, st);
 }
 
 // ---- paged decode attention ---------------------------------------------------------------
@@ -335,24 +387,45 @@ __global__ void __launch_bounds__(kPaSplitKeys) paged_attention_split_kernel(
   }
 }
 
-__global__ void paged_attention_merge_kernel(const float *__restrict__ partial, int n_splits, int d,
-                                             float *__restrict__ out) {
-  const int head = blockIdx.x;
+// Combines the splits of one query head: weights exp(m_s - max m) are formed once per split, then each
+// thread reduces one output dim over the splits (coalesced reads of the partial records).
+constexpr int kPaMergeMaxSplits = 1024;
+__global__ void __launch_bounds__(128) paged_attention_merge_kernel(const float *__restrict__ partial, int n_splits,
+                                                                    int d, float *__restrict__ out) {
+  __shared__ float w_s[kPaMergeMaxSplits];
+  __shared__ float red[4];
+  const int head = blockIdx.x, tid = threadIdx.x;
   const float *rec = partial + (long long)head * n_splits * (d + 2);
-  float mm = -FLT_MAX;
-  for (int s = 0; s < n_splits; ++s) mm = fmaxf(mm, rec[s * (d + 2)]);
+  float mx = -FLT_MAX;
+  for (int s = tid; s < n_splits; s += 128) mx = fmaxf(mx, rec[(long long)s * (d + 2)]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  if ((tid & 31) == 0) red[tid >> 5] = mx;
+  __syncthreads();
+  mx = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
+  __syncthreads();
   float ll = 0.f;
-  for (int s = 0; s < n_splits; ++s) ll += rec[s * (d + 2) + 1] * __expf(rec[s * (d + 2)] - mm);
-  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+  for (int s = tid; s < n_splits; s += 128) {
+    const float wgt = __expf(rec[(long long)s * (d + 2)] - mx);
+    w_s[s] = wgt;
+    ll += rec[(long long)s * (d + 2) + 1] * wgt;
+  }
+  ll = warp_sum_d(ll);
+  if ((tid & 31) == 0) red[tid >> 5] = ll;
+  __syncthreads();
+  ll = red[0] + red[1] + red[2] + red[3];
+  const float inv = 1.f / ll;
+  for (int c = tid; c < d; c += 128) {
     float a = 0.f;
-    for (int s = 0; s < n_splits; ++s) a += rec[s * (d + 2) + 2 + c] * __expf(rec[s * (d + 2)] - mm);
-    out[head * d + c] = a / ll;
+    for (int s = 0; s < n_splits; ++s) a += rec[(long long)s * (d + 2) + 2 + c] * w_s[s];
+    out[head * d + c] = a * inv;
   }
 }
 
 int paged_attention(const float *q, int n_q_heads, CacheView cache, int layer, const int *block_table_dev,
                     int n_ctx, void *scratch, float *out, cudaStream_t st) {
   const int splits = pa_splits(n_ctx);
+  if (splits > kPaMergeMaxSplits) return KV_ERR_SHAPE;   // 262,144 context tokens
   const dim3 grid(cache.n_kv_heads, splits);
   float *partial = (float *)scratch;
   if (cache.head_dim == 64)
