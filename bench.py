@@ -35,6 +35,11 @@ FALLBACK_BF16_TFLOPS_SUSTAINED = 1400.0
 WORKLOADS = {
     # name: (shape, prefix tokens, suffix tokens, pool blocks)
     "32b-4k": ("32b", 4096, 512, 4096),
+    # prefix-length sweep of the same shape, suffix = prefix / 8 (parity cases / context; not the bench line)
+    "32b-512": ("32b", 512, 64, 4096),
+    "32b-2k": ("32b", 2048, 256, 4096),
+    "32b-8k": ("32b", 8192, 1024, 4096),
+    "32b-16k": ("32b", 16384, 2048, 4096),
     "8b-1k": ("8b", 1024, 256, 1024),
     "tiny": ("tiny", 128, 32, 64),
 }
@@ -186,6 +191,7 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
     import paper_2608_16477_b200 as kv
+    from paper_2608_16477_b200 import replicas
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -272,12 +278,7 @@ def run_ours(args):
             fn()
         e1.record(stream)
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return replicas.max_over_ranks(e0.elapsed_time(e1), device="cuda")
 
     # standalone pack / unpack bandwidth, rotating over disjoint block sets so every launch reads cold pages.
     # Timed alone, before the compute-heavy steps pull the clocks down under the power cap: the same condition
@@ -343,7 +344,7 @@ def run_ours(args):
 
     pk = peaks()
     ms_per_step = total_ms / args.steps
-    value = world * prefix / (ms_per_step * 1e-3)
+    value = replicas.whole_job_throughput(prefix, world, ms_per_step)
     per_step = {k: (ms / args.steps, cnt // args.steps) for k, (ms, cnt) in prof.items()}
     prefill_kinds = ("embed", "rmsnorm", "gemm_qkv", "rope_store", "attention", "gemm_o", "gemm_gate_up", "gemm_down")
     prefill_ms = sum(per_step[k][0] for k in prefill_kinds)

@@ -358,6 +358,9 @@ int32_t kv_prefill_prefix(kv_model *m, const kv_cache_desc *cache, const int32_t
     if (rc__ != KV_OK) return rc__; \
   } while (0)
   { ProfScope ps(PROF_ROPE_STORE, st); KV_TRY(rope_table(w.rope, pos0, t, d.head_dim, d.rope_base, st)); }
+  // the qkv buffer has one row per context position; the chunk's rows start at pos0
+  const bool tc_attention = attention_tc_supported(d.n_q_heads, d.n_kv_heads, d.head_dim);
+  bf16 *qkv_chunk = w.qkv + (long long)pos0 * qkv_dim;
   { ProfScope ps(PROF_EMBED, st); KV_TRY(embed_rows(m->embed, w.ids, t, d.hidden, w.x, st)); }
   for (int l = 0; l < d.n_layers; ++l) {
     { ProfScope ps(PROF_RMSNORM, st); KV_TRY(rmsnorm_rows(w.x, m->attn_norm[l], t, d.hidden, d.rms_eps, w.h, st)); }
@@ -372,11 +375,20 @@ int32_t kv_prefill_prefix(kv_model *m, const kv_cache_desc *cache, const int32_t
       qa.n_q_heads = d.n_q_heads;
       qa.n_kv_heads = d.n_kv_heads;
       qa.layer = l;
-      KV_TRY(run_gemm(m, w.h, d.hidden, m->w_qkv[l], t, qkv_dim, d.hidden, GEMM_QKV_ROPE, w.qkv, nullptr, w.status, st, &qa));
+      KV_TRY(run_gemm(m, w.h, d.hidden, m->w_qkv[l], t, qkv_dim, d.hidden, GEMM_QKV_ROPE, qkv_chunk, nullptr, w.status, st, &qa));
     }
     if (l == d.n_layers - 1 && logits_out_dev == nullptr) break;   // K/V of the last layer are complete
-    { ProfScope ps(PROF_ATTENTION, st); KV_TRY(attention_prefill(w.qkv, t, pos0, d.n_q_heads, d.n_kv_heads, d.head_dim, cv, l, w.table, w.attn,
-                             reinterpret_cast<int *>(w.status), st)); }
+    {
+      ProfScope ps(PROF_ATTENTION, st);
+      if (tc_attention) {
+        KV_TRY(gather_prefix_kv(w.qkv, pos0, d.n_q_heads, d.n_kv_heads, d.head_dim, cv, l, w.table, st));
+        KV_TRY(attention_prefill_tc(w.qkv, t, pos0, d.n_q_heads, d.n_kv_heads, d.head_dim, w.attn,
+                                    reinterpret_cast<int *>(w.status), st));
+      } else {
+        KV_TRY(attention_prefill(qkv_chunk, t, pos0, d.n_q_heads, d.n_kv_heads, d.head_dim, cv, l, w.table, w.attn,
+                                 reinterpret_cast<int *>(w.status), st));
+      }
+    }
     { ProfScope ps(PROF_GEMM_O, st); KV_TRY(run_gemm(m, w.attn, q_dim, m->w_o[l], t, d.hidden, q_dim, GEMM_RESID_F32, nullptr, w.x, w.status, st)); }
     { ProfScope ps(PROF_RMSNORM, st); KV_TRY(rmsnorm_rows(w.x, m->ffn_norm[l], t, d.hidden, d.rms_eps, w.h, st)); }
     { ProfScope ps(PROF_GEMM_GATE_UP, st); KV_TRY(run_gemm(m, w.h, d.hidden, m->w_gate_up[l], t, d.ffn, d.hidden, GEMM_SWIGLU, w.mid, nullptr, w.status, st)); }

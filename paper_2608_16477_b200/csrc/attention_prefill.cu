@@ -3,9 +3,10 @@
 // Query rows are the chunk's positions pos0 .. pos0+T-1; keys/values of the chunk come from the
 // contiguous post-RoPE qkv buffer, earlier positions [0,pos0) from the paged cache through the block
 // table.  Online softmax in fp32 (running max / sum), outputs bf16.
-// A fresh prefill (pos0 = 0) with head_dim 64/128 and an even number of query heads per KV head runs on the
-// tensor-core kernel (attention_tcgen05.cu).  The kernel below serves continued prefill (pos0 > 0, keys
-// read from pages) and the remaining head layouts.
+// head_dim 64/128 with an even number of query heads per KV head runs on the tensor-core kernel
+// (attention_tcgen05.cu); the prefill path gathers a cached prefix into the qkv buffer for it.  The kernel
+// below reads earlier positions straight from the pages and serves the remaining head layouts and the
+// single-kernel entry point with pos0 > 0.
 #include <float.h>
 
 #include "common.cuh"
@@ -96,15 +97,13 @@ __global__ void __launch_bounds__(kApWarps * 32) attention_prefill_simt_kernel(
     if (i < dpl) orow[lane + 32 * i] = __float2bfloat16_rn(acc[i] * inv);
 }
 
-int attention_prefill_tc(const bf16 *qkv, int n_tokens, int n_q_heads, int n_kv_heads, int head_dim, bf16 *out,
-                         int *status_dev, cudaStream_t st);
 
 int attention_prefill(const bf16 *qkv, int n_tokens, int pos0, int n_q_heads, int n_kv_heads, int head_dim,
                       CacheView cache, int layer, const int *block_table_dev, bf16 *out, int *status_dev,
                       cudaStream_t st) {
   if (n_tokens <= 0) return KV_OK;
-  if (pos0 == 0 && (head_dim == 64 || head_dim == 128) && ((n_q_heads / n_kv_heads) % 2 == 0))
-    return attention_prefill_tc(qkv, n_tokens, n_q_heads, n_kv_heads, head_dim, out, status_dev, st);
+  if (pos0 == 0 && attention_tc_supported(n_q_heads, n_kv_heads, head_dim))
+    return attention_prefill_tc(qkv, n_tokens, 0, n_q_heads, n_kv_heads, head_dim, out, status_dev, st);
   dim3 grid((n_tokens + kApWarps - 1) / kApWarps, n_q_heads);
   attention_prefill_simt_kernel<<<grid, kApWarps * 32, 0, st>>>(qkv, n_tokens, pos0, n_q_heads, n_kv_heads,
                                                                head_dim, cache, layer, block_table_dev, out);

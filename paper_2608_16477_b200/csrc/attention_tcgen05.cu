@@ -1,4 +1,6 @@
-// Causal GQA flash attention for prefill on the 5th-generation tensor cores (pos0 = 0, head_dim 64 or 128).
+// Causal GQA flash attention for prefill on the 5th-generation tensor cores (head_dim 64 or 128).
+// The qkv buffer holds one row per context position: rows [0, pos0) carry the K/V of an already cached
+// prefix (gathered from its pages), rows [pos0, pos0 + T) the chunk's post-RoPE Q, K and V.
 //
 // One CTA works on ONE 128-row query tile of TWO query heads that share a KV head (tiles "a" and "b"), so
 // every K/V tile fetched by TMA feeds both, and the two softmax warpgroups alternate with the tensor core:
@@ -81,8 +83,8 @@ struct AttnSmem {
 
 template <int D>
 __global__ void __launch_bounds__(kAttnThreads, 1)
-attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_tokens, int n_q_heads, int n_kv_heads,
-                            float scale_log2, bf16 *__restrict__ out, DeviceStatus *status) {
+attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_tokens, int pos0, int n_q_heads,
+                            int n_kv_heads, float scale_log2, bf16 *__restrict__ out, DeviceStatus *status) {
   using L = AttnSmem<D>;
   constexpr int kAtoms = D / 64;                   // 64-column (128-byte) boxes per tile row
   constexpr int kBoxBytes = kBM * 128;             // one 128-row x 64-col box
@@ -104,8 +106,10 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
   const int pair = blockIdx.x % pairs;
   const int head_a = 2 * pair, head_b = head_a + 1;
   const int kv_head = head_a / group;
-  const int m0 = m_tile * kBM;
-  const int n_kv = m_tile + 1;                                     // causal: key tiles 0 .. m_tile
+  const int m0 = m_tile * kBM;                                     // first chunk row of this tile
+  const int n_ctx = pos0 + n_tokens;
+  // causal: key tiles up to the one holding the last row's own position
+  const int n_kv = min((n_ctx + kBN - 1) / kBN, (pos0 + m0 + kBM - 1) / kBN + 1);
   const int q_col[2] = {head_a * D, head_b * D};
   const int k_col = (n_q_heads + kv_head) * D;
   const int v_col = (n_q_heads + n_kv_heads + kv_head) * D;
@@ -139,7 +143,7 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
       for (int t = 0; t < 2; ++t) {
         tc::mbar_expect_tx(bar(B_Q, t), L::kTileBytes);
         for (int a = 0; a < kAtoms; ++a)
-          tc::tma_load_2d(smem_base + L::kQOff + t * L::kTileBytes + a * kBoxBytes, &tma_qkv, q_col[t] + a * 64, m0,
+          tc::tma_load_2d(smem_base + L::kQOff + t * L::kTileBytes + a * kBoxBytes, &tma_qkv, q_col[t] + a * 64, pos0 + m0,
                           bar(B_Q, t));
       }
       for (int j = 0; j < n_kv; ++j) {
@@ -215,7 +219,7 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
     const int t = (warp - 4) >> 2;                 // 0: tile a, 1: tile b
     const int quarter = warp & 3;
     const int row_in_tile = quarter * 32 + lane;
-    const int qi = m0 + row_in_tile;               // absolute query position (pos0 = 0)
+    const int qi = pos0 + m0 + row_in_tile;        // absolute query position
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
     const uint32_t s_t = tmem_base + lane_base + (t == 0 ? kTmemS0 : kTmemS1);
     const uint32_t o_t = tmem_base + lane_base + (t == 0 ? kTmemO0 : kTmemO1);
@@ -226,7 +230,7 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc::tc_fence_after();
-      const bool diag = (j == n_kv - 1);
+      const bool diag = (j * kBN + kBN - 1 > pos0 + m0);   // tile reaches past the first row's position
       const int limit = qi - j * kBN;              // keys with column > limit are masked
       // the whole row of S (128 fp32) in registers: four loads in flight, one wait
       uint32_t r0[32], r1[32], r2[32], r3[32];
@@ -308,13 +312,14 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
       tc::tc_fence_after();
       const float inv = 1.f / l_sum;
       const int head = (t == 0) ? head_a : head_b;
-      bf16 *orow = out + (long long)qi * n_q_heads * D + head * D;
+      const int out_row = m0 + row_in_tile;        // row inside the chunk
+      bf16 *orow = out + (long long)out_row * n_q_heads * D + head * D;
 #pragma unroll 1
       for (int c = 0; c < D / 32; ++c) {
         uint32_t r[32];
         tc::tmem_ld32(o_t + c * 32, r);
         tc::tmem_ld_wait();
-        if (qi < n_tokens) {
+        if (out_row < n_tokens) {
           uint4 *dst = reinterpret_cast<uint4 *>(orow + c * 32);
 #pragma unroll
           for (int v = 0; v < 4; ++v)
@@ -337,13 +342,44 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
 
 }  // namespace
 
-// pos0 == 0, head_dim 64 or 128, even number of query heads per KV head.
-int attention_prefill_tc(const bf16 *qkv, int n_tokens, int n_q_heads, int n_kv_heads, int head_dim, bf16 *out,
-                         int *status_dev, cudaStream_t st) {
+// Copies the cached prefix's K and V (positions [0, pos0)) of one layer from their pages into rows [0, pos0)
+// of the qkv buffer, so the attention kernel's TMA map covers the whole context with one row pitch.
+__global__ void __launch_bounds__(128) gather_prefix_kv_kernel(bf16 *__restrict__ qkv, int qkv_dim, int k_col,
+                                                               int v_col, CacheView cache, int layer,
+                                                               const int *__restrict__ block_table) {
+  const int pos = blockIdx.x;
+  const int block = block_table[pos / cache.block_size];
+  const long long off = (long long)(pos % cache.block_size) * cache.n_kv_heads * cache.head_dim;
+  const int vecs = cache.n_kv_heads * cache.head_dim / 8;
+  const uint4 *ksrc = reinterpret_cast<const uint4 *>(reinterpret_cast<const bf16 *>(cache.page(layer, 0, block)) + off);
+  const uint4 *vsrc = reinterpret_cast<const uint4 *>(reinterpret_cast<const bf16 *>(cache.page(layer, 1, block)) + off);
+  uint4 *kdst = reinterpret_cast<uint4 *>(qkv + (long long)pos * qkv_dim + k_col);
+  uint4 *vdst = reinterpret_cast<uint4 *>(qkv + (long long)pos * qkv_dim + v_col);
+  for (int v = threadIdx.x; v < vecs; v += blockDim.x) {
+    kdst[v] = ksrc[v];
+    vdst[v] = vsrc[v];
+  }
+}
+
+int gather_prefix_kv(bf16 *qkv_ctx, int pos0, int n_q_heads, int n_kv_heads, int head_dim, CacheView cache, int layer,
+                     const int *block_table_dev, cudaStream_t st) {
+  if (pos0 <= 0) return KV_OK;
+  const int qkv_dim = (n_q_heads + 2 * n_kv_heads) * head_dim;
+  gather_prefix_kv_kernel<<<pos0, 128, 0, st>>>(qkv_ctx, qkv_dim, n_q_heads * head_dim,
+                                                (n_q_heads + n_kv_heads) * head_dim, cache, layer, block_table_dev);
+  KV_COUNT_LAUNCH();
+  KV_CUDA(cudaGetLastError());
+  return KV_OK;
+}
+
+// head_dim 64 or 128, even number of query heads per KV head.  qkv_ctx has pos0 + n_tokens rows (see the file
+// header); out has n_tokens rows.
+int attention_prefill_tc(const bf16 *qkv_ctx, int n_tokens, int pos0, int n_q_heads, int n_kv_heads, int head_dim,
+                         bf16 *out, int *status_dev, cudaStream_t st) {
   if (n_tokens <= 0) return KV_OK;
   const int qkv_dim = (n_q_heads + 2 * n_kv_heads) * head_dim;
   CUtensorMap map;
-  int rc = tc::make_tmap_2d(&map, qkv, n_tokens, qkv_dim, qkv_dim, kBM);
+  int rc = tc::make_tmap_2d(&map, qkv_ctx, pos0 + n_tokens, qkv_dim, qkv_dim, kBM);
   if (rc != KV_OK) return rc;
   static bool attr_set = false;
   if (!attr_set) {
@@ -358,10 +394,10 @@ int attention_prefill_tc(const bf16 *qkv, int n_tokens, int n_q_heads, int n_kv_
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)head_dim);
   DeviceStatus *status = reinterpret_cast<DeviceStatus *>(status_dev);
   if (head_dim == 64)
-    attention_prefill_tc_kernel<64><<<grid, kAttnThreads, AttnSmem<64>::kBytes, st>>>(map, n_tokens, n_q_heads,
+    attention_prefill_tc_kernel<64><<<grid, kAttnThreads, AttnSmem<64>::kBytes, st>>>(map, n_tokens, pos0, n_q_heads,
                                                                                      n_kv_heads, scale_log2, out, status);
   else
-    attention_prefill_tc_kernel<128><<<grid, kAttnThreads, AttnSmem<128>::kBytes, st>>>(map, n_tokens, n_q_heads,
+    attention_prefill_tc_kernel<128><<<grid, kAttnThreads, AttnSmem<128>::kBytes, st>>>(map, n_tokens, pos0, n_q_heads,
                                                                                        n_kv_heads, scale_log2, out, status);
   KV_COUNT_LAUNCH();
   KV_CUDA(cudaGetLastError());

@@ -80,6 +80,13 @@ int gemm_simt(const bf16 *a, int lda, const bf16 *w, int m, int n, int k, int mo
 int embed_rows(const bf16 *embed, const int *ids_dev, int n_tokens, int hidden, float *x, cudaStream_t st);
 int rmsnorm_rows(const float *x, const bf16 *gain, int rows, int dim, float eps, bf16 *out, cudaStream_t st);
 int rope_table(float2 *table, int pos0, int n_tokens, int head_dim, float base, cudaStream_t st);
+inline bool attention_tc_supported(int n_q_heads, int n_kv_heads, int head_dim) {
+  return (head_dim == 64 || head_dim == 128) && ((n_q_heads / n_kv_heads) % 2 == 0);
+}
+int attention_prefill_tc(const bf16 *qkv_ctx, int n_tokens, int pos0, int n_q_heads, int n_kv_heads, int head_dim,
+                         bf16 *out, int *status_dev, cudaStream_t st);
+int gather_prefix_kv(bf16 *qkv_ctx, int pos0, int n_q_heads, int n_kv_heads, int head_dim, CacheView cache, int layer,
+                     const int *block_table_dev, cudaStream_t st);
 int attention_prefill(const bf16 *qkv, int n_tokens, int pos0, int n_q_heads, int n_kv_heads,
                       int head_dim, CacheView cache, int layer, const int *block_table_dev, bf16 *out,
                       int *status_dev, cudaStream_t st);

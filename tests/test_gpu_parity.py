@@ -120,7 +120,8 @@ def test_pack_unpack_batched_pattern_32b_pages(kv, torch):
 
 
 # ------------------------------------------------------------------ single kernels
-@pytest.mark.parametrize("m,n,k", [(128, 256, 64), (300, 520, 192), (1000, 1048, 512), (16, 8, 64), (257, 1280, 1024)])
+@pytest.mark.parametrize("m,n,k", [(128, 256, 64), (300, 520, 192), (1000, 1048, 512), (16, 8, 64), (257, 1280, 1024),
+                                   (512, 25600, 256), (512, 4736, 128), (1024, 12288, 64)])
 @pytest.mark.parametrize("mode", [0, 1, 2])
 def test_gemm_tensor_core(kv, torch, m, n, k, mode):
     rng = np.random.default_rng(100 + m + n + k + mode)
@@ -307,3 +308,35 @@ def test_chunked_prefill_matches_single_shot(kv, torch):
     b = O.from_bf16_bits(two.as_logical_numpy()).astype(np.float64)
     st = error_stats(b, a)
     assert st["rel_l2"] <= 5e-3, st
+
+
+def test_chunked_prefill_wide_shape_tensor_core_path(kv, torch):
+    """Continued prefill in 256-token chunks (the chunk size the paper uses under contention, Section 6.5) on a
+    32B-shaped two-layer model: the cached prefix is gathered for the tensor-core attention kernel.  The result
+    must agree with the single-shot prefill up to the ulp flips a different tile split of the same sums causes."""
+    s = synth.SHAPES["32b"].with_layers(2)
+    s = synth.ModelShape(**{**s.__dict__, "vocab": 2048})
+    n = 1000                                           # ragged: last chunk has 232 tokens
+    ids = synth.token_ids(s, 5, n)
+    head = synth.head_weights(s, 5)
+    model = kv.Model(s, head, lambda l: synth.layer_weights(s, 5, l))
+    table = synth.block_permutation(6, 128)[: -(-n // 16)]
+    one = kv.PagedCache(s, 128, fill=0)
+    two = kv.PagedCache(s, 128, fill=0)
+    lg1 = torch.empty(s.vocab, dtype=torch.float32, device="cuda")
+    lg2 = torch.empty(s.vocab, dtype=torch.float32, device="cuda")
+    ws = kv.kv_prefill_prefix(model, one, ids, table, logits_out=lg1)
+    kv.kv_check_device_status(ws)
+    for p0 in range(0, n, 256):
+        chunk = ids[p0:p0 + 256]
+        last = p0 + 256 >= n
+        ws = kv.kv_prefill_prefix(model, two, chunk, table[: -(-(p0 + len(chunk)) // 16)], pos0=p0,
+                                  logits_out=lg2 if last else None)
+        kv.kv_check_device_status(ws)
+    torch.cuda.synchronize()
+    a = O.from_bf16_bits(one.as_logical_numpy()).astype(np.float64)
+    b = O.from_bf16_bits(two.as_logical_numpy()).astype(np.float64)
+    st = error_stats(b, a)
+    sl = error_stats(lg2.cpu().numpy(), lg1.cpu().numpy())
+    print("chunked vs single-shot:", st, sl)
+    assert st["rel_l2"] <= 5e-3 and sl["rel_l2"] <= 1e-2, (st, sl)
