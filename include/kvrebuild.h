@@ -193,6 +193,13 @@ int32_t kv_unpack_blocks_batched(const kv_cache_desc *dst, int32_t n_req, const 
 int32_t kv_op_gemm(const void *a_dev, int32_t lda, const void *w_dev, int32_t m, int32_t n, int32_t k,
                    int32_t mode, void *out_dev, float *resid_dev, int32_t *status_dev, void *stream);
 
+/* Matrix-vector product of the decode step: W bf16 [rows, k] row-major, x fp32 [k], y fp32.
+ * mode 0: y[n] = W[n] . x (n rows).  mode 1: y[n] += W[n] . x.  mode 2: W is [2n, k] (gate | up),
+ * y[n] = silu(W[n] . x) * (W[n + n_rows] . x).  gain_dev != NULL (bf16 [k], modes 0 and 2) fuses the preceding
+ * RMSNorm: x is replaced by x * gain * rsqrt(mean(x^2) + eps).  k must be a multiple of 8. */
+int32_t kv_op_gemv(const void *w_dev, const float *x_dev, int32_t n, int32_t k, int32_t mode, const void *gain_dev,
+                   float eps, float *y_dev, void *stream);
+
 /* Diagnostics.  The same projection computed by a plain CUDA-core kernel (no tensor cores, no TMA):
  * an independent on-device cross-check of kv_op_gemm for unit tests.  No operation above uses it. */
 int32_t kv_op_gemm_reference(const void *a_dev, int32_t lda, const void *w_dev, int32_t m, int32_t n, int32_t k,

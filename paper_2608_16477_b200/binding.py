@@ -19,7 +19,7 @@ EXPORTS = [
     "kv_unpack_assemble", "kv_decode_step", "kv_pack_blocks_batched", "kv_unpack_blocks_batched",
     "kv_op_gemm", "kv_op_gemm_reference", "kv_op_rmsnorm",
     "kv_op_attention_prefill", "kv_paged_attention_scratch_bytes", "kv_op_paged_attention", "kv_fill_pattern",
-    "kv_profile_enable", "kv_profile_read", "kv_launch_count", "kv_op_paged_attention_noalloc", "kv_check_copy_status",
+    "kv_profile_enable", "kv_profile_read", "kv_launch_count", "kv_op_paged_attention_noalloc", "kv_check_copy_status", "kv_op_gemv",
 ]
 
 PROFILE_KINDS = ("embed", "rmsnorm", "gemm_qkv", "rope_store", "attention", "gemm_o", "gemm_gate_up", "gemm_down",
@@ -96,6 +96,7 @@ def load(build_if_missing: bool = True):
         "kv_fill_pattern": (i32, [vp, i64, C.c_uint64, i64, vp]),
         "kv_op_paged_attention_noalloc": (i32, [vp, i32, C.POINTER(CacheDesc), i32, vp, i32, vp, vp]),
         "kv_check_copy_status": (i32, [vp]),
+        "kv_op_gemv": (i32, [vp, vp, i32, i32, i32, vp, C.c_float, vp, vp]),
         "kv_profile_enable": (i32, [i32]),
         "kv_profile_read": (i32, [C.POINTER(C.c_float), C.POINTER(C.c_int64), i32]),
         "kv_launch_count": (i64, []),
@@ -369,3 +370,9 @@ def kv_op_paged_attention_noalloc(q, cache: PagedCache, layer, block_table_dev, 
 
 def kv_check_copy_status(stream=None) -> None:
     _check(load().kv_check_copy_status(_stream(stream)), "kv_check_copy_status")
+
+
+def kv_op_gemv(w, x, mode: int, y, gain=None, eps: float = 0.0, stream=None, n=None):
+    rows, k = w.shape
+    n = n if n is not None else (rows // 2 if mode == 2 else rows)
+    _check(load().kv_op_gemv(_ptr(w), _ptr(x), n, k, mode, _ptr(gain), eps, _ptr(y), _stream(stream)), "kv_op_gemv")

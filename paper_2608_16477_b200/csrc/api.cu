@@ -548,6 +548,16 @@ int32_t kv_op_gemm_reference(const void *a_dev, int32_t lda, const void *w_dev, 
                    (cudaStream_t)stream);
 }
 
+int32_t kv_op_gemv(const void *w_dev, const float *x_dev, int32_t n, int32_t k, int32_t mode, const void *gain_dev,
+                   float eps, float *y_dev, void *stream) {
+  if (w_dev == nullptr || x_dev == nullptr || y_dev == nullptr || n <= 0 || k <= 0 || mode < 0 || mode > 2)
+    return KV_ERR_ARG;
+  if (((uintptr_t)w_dev & 15) || ((uintptr_t)x_dev & 15) || (gain_dev != nullptr && ((uintptr_t)gain_dev & 15)))
+    return KV_ERR_ARG;
+  if (gain_dev != nullptr && mode == 1) return KV_ERR_ARG;
+  return gemv((const bf16 *)w_dev, x_dev, n, k, mode, y_dev, (cudaStream_t)stream, (const bf16 *)gain_dev, eps);
+}
+
 int32_t kv_op_rmsnorm(const float *x_dev, const void *gain_dev, int32_t rows, int32_t dim, float eps, void *out_dev,
                       void *stream) {
   if (x_dev == nullptr || gain_dev == nullptr || out_dev == nullptr || rows < 0 || dim <= 0 || dim % 4 != 0)

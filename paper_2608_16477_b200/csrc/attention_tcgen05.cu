@@ -30,8 +30,12 @@ constexpr int kKvStages = 2;
 constexpr int kAttnThreads = 384;   // 12 warps
 constexpr uint32_t kTmemS0 = 0, kTmemS1 = 128, kTmemO0 = 256, kTmemO1 = 384;
 constexpr float kRescaleThreshold = 8.0f;
+// setmaxnreg moves registers inside the pool the CTA was launched with (threads x registers per thread as
+// compiled), and setmaxnreg.inc blocks, with no timeout, until the registers it asks for have been released.
+// The launcher therefore checks 256 x (kRegsSoftmax - compiled) <= 128 x (compiled - kRegsOther) before the
+// first launch and refuses to launch otherwise (compiled = 168 here: 256 x 48 = 128 x 96).
 constexpr int kRegsOther = 72;      // registers per thread of warps 0-3 after the hand-back
-constexpr int kRegsSoftmax = 216;   // registers per thread of the softmax warps (128 x 72 + 256 x 216 <= 64 Ki)
+constexpr int kRegsSoftmax = 216;   // registers per thread of the softmax warps
 
 enum AttnTag { ATAG_Q = 11, ATAG_KV_EMPTY = 12, ATAG_K = 13, ATAG_V = 14, ATAG_S = 15, ATAG_P = 16, ATAG_O = 17 };
 
@@ -381,14 +385,25 @@ int attention_prefill_tc(const bf16 *qkv_ctx, int n_tokens, int pos0, int n_q_he
   CUtensorMap map;
   int rc = tc::make_tmap_2d(&map, qkv_ctx, pos0 + n_tokens, qkv_dim, qkv_dim, kBM);
   if (rc != KV_OK) return rc;
-  static bool attr_set = false;
-  if (!attr_set) {
+  static int regs_ok = -1;
+  if (regs_ok < 0) {
     KV_CUDA(cudaFuncSetAttribute(attention_prefill_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  AttnSmem<64>::kBytes));
     KV_CUDA(cudaFuncSetAttribute(attention_prefill_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  AttnSmem<128>::kBytes));
-    attr_set = true;
+    // the register hand-over must balance inside the CTA's own pool, or setmaxnreg.inc would wait forever
+    regs_ok = 1;
+    cudaFuncAttributes fa;
+    KV_CUDA(cudaFuncGetAttributes(&fa, attention_prefill_tc_kernel<64>));
+    const int r64 = fa.numRegs;
+    KV_CUDA(cudaFuncGetAttributes(&fa, attention_prefill_tc_kernel<128>));
+    const int r128 = fa.numRegs;
+    for (int compiled : {r64, r128}) {
+      const int softmax_threads = kAttnThreads - 128;
+      if (compiled < kRegsOther || softmax_threads * (kRegsSoftmax - compiled) > 128 * (compiled - kRegsOther)) regs_ok = 0;
+    }
   }
+  if (regs_ok == 0) return KV_ERR_SHAPE;
   const int m_tiles = (n_tokens + kBM - 1) / kBM;
   const int grid = m_tiles * (n_q_heads / 2);
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)head_dim);

@@ -75,11 +75,17 @@ def main():
                 kv.kv_unpack_assemble(cache, wires[i], np.arange(a.blocks), ids, [], a.blocks * s.block_size)
         work, unit = 2.0 * a.blocks * s.n_layers * 2 * cache.page_bytes / 1e9, "GB/s"
     elif a.case == "decode_gemv":
-        w = rnd(2 * s.ffn, s.hidden, std=0.02)
+        # the gate/up product of one decode step (524 MB of weights), rotating over 4 weight copies (> L2)
+        ws = [rnd(2 * s.ffn, s.hidden, std=0.02) for _ in range(4)]
         x = torch.randn(s.hidden, device=dev)
+        gain = torch.ones(s.hidden, dtype=torch.bfloat16, device=dev)
         y = torch.empty(s.ffn, device=dev)
-        lib = kv.load()
-        raise SystemExit("decode_gemv has no single-kernel entry point; profile bench.py instead")
+        state = {"i": 0}
+
+        def run():
+            state["i"] += 1
+            kv.kv_op_gemv(ws[state["i"] % 4], x, 2, y, gain=gain, eps=1e-6)
+        work, unit = ws[0].numel() * 2 / 1e9, "GB/s"
     else:
         raise SystemExit(f"unknown case {a.case}")
     run()

@@ -164,6 +164,25 @@ def test_gemm_matches_cuda_core_crosscheck(kv, torch):
     assert torch.max(torch.abs(o1.float() - o2.float())).item() <= 2.0 ** -7 * torch.max(torch.abs(o2.float())).item()
 
 
+@pytest.mark.parametrize("n,k", [(37, 256), (512, 5120), (1001, 1064)])
+@pytest.mark.parametrize("mode,norm", [(0, False), (0, True), (1, False), (2, False), (2, True)])
+def test_gemv_decode(kv, torch, n, k, mode, norm):
+    rng = np.random.default_rng(n + k + mode)
+    rows = 2 * n if mode == 2 else n
+    w = synth.bf16_round_f32(rng.standard_normal((rows, k), dtype=np.float32) / np.float32(np.sqrt(k)))
+    x = (rng.standard_normal(k) * 2.0).astype(np.float32)
+    g = synth.bf16_round_f32(rng.uniform(0.5, 1.5, k).astype(np.float32))
+    y0 = rng.standard_normal(n).astype(np.float32)
+    xin = O.rmsnorm(x[None], g, 1e-6)[0] if norm else x.astype(np.float64)
+    prod = w.astype(np.float64) @ xin
+    want = prod if mode == 0 else (y0 + prod if mode == 1 else O.silu(prod[:n]) * prod[n:])
+    y = torch.from_numpy(y0.copy()).cuda()
+    kv.kv_op_gemv(torch.from_numpy(w).cuda().to(torch.bfloat16), torch.from_numpy(x).cuda(), mode, y,
+                  gain=torch.from_numpy(g).cuda().to(torch.bfloat16) if norm else None, eps=1e-6)
+    got = y.cpu().numpy()
+    assert np.max(np.abs(got - want)) <= 2e-5 * np.sqrt(k) * max(1.0, np.max(np.abs(want))), error_stats(got, want)
+
+
 def test_rmsnorm_rows(kv, torch):
     rng = np.random.default_rng(6)
     x = (rng.standard_normal((37, 5120)) * 3).astype(np.float32)
