@@ -30,17 +30,27 @@ constexpr int kTmemCols = 512;
 constexpr int kTmemBufStride = 256;             // the two accumulators sit at columns 0 and 256
 constexpr int kThreads = 192;
 constexpr int kMaxSmem = 232448;                // 227 KiB per CTA
+constexpr int kEpiStageBytes = 4 * 32 * 8 * 4;  // per epilogue warp: a 32-row x 8-column fp32 transpose buffer (1 KiB)
 
 // Tile width BN (accumulator columns) is a template parameter: 256 by default, narrower tiles where they
 // remove a mostly empty last wave (e.g. N = 5120 over 148 SMs: 23 tiles of 224 fill 4.97 waves, 20 of 256 need 5 of 4.3).
-template <int BN>
+template <int MODE, int BN>
 struct TileCfg {
   static constexpr int kBBytes = BN * BK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kStagesFit = (kMaxSmem - 1024 - 256) / kStageBytes;
+  static constexpr int kEpiBytes = (MODE == GEMM_RESID_F32) ? kEpiStageBytes : 0;
+  static constexpr int kStagesFit = (kMaxSmem - 1024 - 256 - kEpiBytes) / kStageBytes;
   static constexpr int kStages = kStagesFit > 6 ? 6 : kStagesFit;
-  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + kEpiBytes;
 };
+
+#ifdef KV_GEMM_TRACE
+__device__ long long g_gemm_trace[64 * 8];
+#define KV_TRACE(slot, idx) \
+  do { if (blockIdx.x == 0 && (idx) < 64) g_gemm_trace[(idx) * 8 + (slot)] = clock64(); } while (0)
+#else
+#define KV_TRACE(slot, idx) do { } while (0)
+#endif
 
 enum WaitTag { TAG_EMPTY = 1, TAG_FULL = 2, TAG_TMEM_EMPTY = 3, TAG_TMEM_FULL = 4 };
 
@@ -64,9 +74,9 @@ __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CUtensorMap tma_b, int m, int n,
                int k, bf16 *__restrict__ out, float *__restrict__ resid, DeviceStatus *status,
                const __grid_constant__ QkvRopeArgs qa) {
-  constexpr int kStages = TileCfg<BN>::kStages;
-  constexpr int kBBytes = TileCfg<BN>::kBBytes;
-  constexpr int kStageBytes = TileCfg<BN>::kStageBytes;
+  constexpr int kStages = TileCfg<MODE, BN>::kStages;
+  constexpr int kBBytes = TileCfg<MODE, BN>::kBBytes;
+  constexpr int kStageBytes = TileCfg<MODE, BN>::kStageBytes;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t *smem_gen = smem_raw + (smem_base - tc::smem_u32(smem_raw));
@@ -115,6 +125,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
         const int m0 = (tile % m_tiles) * BM;
         const int n0 = (tile / m_tiles) * kOutCols;
+        KV_TRACE(0, (tile - (int)blockIdx.x) / (int)gridDim.x);
         for (int kb = 0; kb < k_blocks; ++kb) {
           ok = tc::mbar_wait(empty_bar(stage), phase ^ 1, abort_flag, status, TAG_EMPTY);
           if (!ok) break;
@@ -143,8 +154,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local) {
         const int buf = local & 1;
         const uint32_t acc_phase = (local >> 1) & 1;
+        KV_TRACE(1, local);
         ok = tc::mbar_wait(tempty_bar(buf), acc_phase ^ 1, abort_flag, status, TAG_TMEM_EMPTY);
         if (!ok) break;
+        KV_TRACE(2, local);
         tc::tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * kTmemBufStride;
         for (int kb = 0; kb < k_blocks; ++kb) {
@@ -161,6 +174,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
           if (++stage == kStages) { stage = 0; phase ^= 1; }
         }
         if (ok) tc::umma_commit(tfull_bar(buf));
+        KV_TRACE(3, local);
       }
     }
   } else {
@@ -173,9 +187,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
       const uint32_t acc_phase = (local >> 1) & 1;
       const int m0 = (tile % m_tiles) * BM;
       const int n0 = (tile / m_tiles) * kOutCols;
+      if (warp == 2 && lane == 0) KV_TRACE(4, local);
       ok = tc::mbar_wait(tfull_bar(buf), acc_phase, abort_flag, status, TAG_TMEM_FULL);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
+      if (warp == 2 && lane == 0) KV_TRACE(5, local);
       tc::tc_fence_after();
       const int row = m0 + quarter * 32 + lane;
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * kTmemBufStride;
@@ -257,6 +273,46 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
               if (col + v * 8 < n) dst[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
           }
         }
+      } else if (MODE == GEMM_RESID_F32) {
+        // x[row, col..] += acc.  A thread owns a row of the accumulator, but rows are 4 * n bytes apart in
+        // memory and a thread-per-row update would touch half a 32-byte sector per row and instruction.
+        // Each warp therefore transposes 32 rows x 8 columns at a time through a 1 KiB shared-memory buffer
+        // and updates x with two lanes per row: every instruction then moves whole 32-byte sectors of 16 rows.
+        float4 *stage = reinterpret_cast<float4 *>(smem_gen + kStages * kStageBytes + 256) + (warp - 2) * 64;
+        const int sub_row = lane >> 1, c4 = lane & 1;
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          const int col = n0 + c * 32;
+          if (col >= n) break;
+          uint32_t r[32];
+          tc::tmem_ld32(t_row + c * 32, r);
+          tc::tmem_ld_wait();
+#pragma unroll
+          for (int s8 = 0; s8 < 4; ++s8) {         // 8 columns per pass
+            const int scol = col + s8 * 8 + c4 * 4;
+            // stage[row][2 chunks], chunk index XORed with bit 2 of the row: conflict-free both ways
+            stage[lane * 2 + (0 ^ ((lane >> 2) & 1))] =
+                make_float4(__uint_as_float(r[8 * s8]), __uint_as_float(r[8 * s8 + 1]), __uint_as_float(r[8 * s8 + 2]),
+                            __uint_as_float(r[8 * s8 + 3]));
+            stage[lane * 2 + (1 ^ ((lane >> 2) & 1))] =
+                make_float4(__uint_as_float(r[8 * s8 + 4]), __uint_as_float(r[8 * s8 + 5]),
+                            __uint_as_float(r[8 * s8 + 6]), __uint_as_float(r[8 * s8 + 7]));
+            __syncwarp();
+#pragma unroll
+            for (int it = 0; it < 2; ++it) {
+              const int rr = it * 16 + sub_row;
+              const int grow = m0 + quarter * 32 + rr;
+              if (grow < m && scol < n) {
+                const float4 a4 = stage[rr * 2 + (c4 ^ ((rr >> 2) & 1))];
+                float4 *px = reinterpret_cast<float4 *>(resid + (long long)grow * n + scol);
+                float4 x = __ldcs(px);
+                x.x += a4.x; x.y += a4.y; x.z += a4.z; x.w += a4.w;
+                *px = x;
+              }
+            }
+            __syncwarp();
+          }
+        }
       } else {
 #pragma unroll 1
         for (int c = 0; c < BN / 32; ++c) {
@@ -265,33 +321,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
           tc::tmem_ld_wait();
           const int col = n0 + c * 32;
           if (row < m && col < n) {
-            if (MODE == GEMM_STORE_BF16) {
-              uint4 *dst = reinterpret_cast<uint4 *>(out + (long long)row * n + col);
+            uint4 *dst = reinterpret_cast<uint4 *>(out + (long long)row * n + col);
 #pragma unroll
-              for (int v = 0; v < 4; ++v)
-                if (col + v * 8 < n)
-                  dst[v] = make_uint4(pack_bf16(__uint_as_float(r[8 * v]), __uint_as_float(r[8 * v + 1])),
-                                      pack_bf16(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3])),
-                                      pack_bf16(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5])),
-                                      pack_bf16(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7])));
-            } else {
-              float4 *dst = reinterpret_cast<float4 *>(resid + (long long)row * n + col);
-#pragma unroll
-              for (int v = 0; v < 8; ++v)
-                if (col + v * 4 < n) {
-                  float4 x = dst[v];
-                  x.x += __uint_as_float(r[4 * v]);
-                  x.y += __uint_as_float(r[4 * v + 1]);
-                  x.z += __uint_as_float(r[4 * v + 2]);
-                  x.w += __uint_as_float(r[4 * v + 3]);
-                  dst[v] = x;
-                }
-            }
+            for (int v = 0; v < 4; ++v)
+              if (col + v * 8 < n)
+                dst[v] = make_uint4(pack_bf16(__uint_as_float(r[8 * v]), __uint_as_float(r[8 * v + 1])),
+                                    pack_bf16(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3])),
+                                    pack_bf16(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5])),
+                                    pack_bf16(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7])));
           }
         }
       }
       tc::tc_fence_before();
       tc::mbar_arrive(tempty_bar(buf));
+      if (warp == 2 && lane == 0) KV_TRACE(6, local);
     }
   }
 
@@ -310,13 +353,13 @@ int launch_gemm(const CUtensorMap &ta, const CUtensorMap &tb, int m, int n, int 
   static bool attr_set = false;
   if (!attr_set) {
     KV_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<MODE, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 TileCfg<BN>::kSmemBytes));
+                                 TileCfg<MODE, BN>::kSmemBytes));
     attr_set = true;
   }
   const int out_cols = (MODE == GEMM_SWIGLU) ? BN / 2 : BN;
   const int tiles = ((m + BM - 1) / BM) * ((n + out_cols - 1) / out_cols);
   const int grid = tiles < sms ? tiles : sms;
-  gemm_tc_kernel<MODE, BN><<<grid, kThreads, TileCfg<BN>::kSmemBytes, st>>>(ta, tb, m, n, k, out, resid, status, qa);
+  gemm_tc_kernel<MODE, BN><<<grid, kThreads, TileCfg<MODE, BN>::kSmemBytes, st>>>(ta, tb, m, n, k, out, resid, status, qa);
   KV_COUNT_LAUNCH();
   KV_CUDA(cudaGetLastError());
   return KV_OK;
@@ -396,5 +439,11 @@ int gemm_tc(const bf16 *a, int lda, const bf16 *w, int m, int n, int k, int mode
 #undef KV_GEMM_CASE
   return KV_ERR_ARG;
 }
+
+#ifdef KV_GEMM_TRACE
+extern "C" int kv_debug_gemm_trace(long long *out_host) {
+  return cudaMemcpyFromSymbol(out_host, g_gemm_trace, sizeof(long long) * 64 * 8) == cudaSuccess ? 0 : -13;
+}
+#endif
 
 }  // namespace kvr

@@ -43,6 +43,9 @@ def main():
         elif a.case == "gemm_o":
             x, w, mode = rnd(t, s.q_dim), rnd(s.hidden, s.q_dim, std=0.02), 1
             out, resid, flops = None, torch.zeros(t, s.hidden, dtype=torch.float32, device=dev), 2.0 * t * s.hidden * s.q_dim
+        elif a.case == "gemm_o_store":          # the O-projection's shape with the plain bf16-store epilogue
+            x, w, mode = rnd(t, s.q_dim), rnd(s.hidden, s.q_dim, std=0.02), 0
+            out, resid, flops = torch.empty(t, s.hidden, dtype=torch.bfloat16, device=dev), None, 2.0 * t * s.hidden * s.q_dim
         elif a.case == "gemm_qkv":
             x, w, mode = rnd(t, s.hidden), rnd(s.qkv_dim, s.hidden, std=0.02), 0
             out, resid, flops = torch.empty(t, s.qkv_dim, dtype=torch.bfloat16, device=dev), None, 2.0 * t * s.hidden * s.qkv_dim
