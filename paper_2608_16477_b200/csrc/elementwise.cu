@@ -45,26 +45,54 @@ int embed_rows(const bf16 *embed, const int *ids_dev, int n_tokens, int hidden, 
 }
 
 // out[r, :] = bf16( x[r, :] * rsqrt(mean(x[r, :]^2) + eps) * gain ), statistics in fp32.
-// One CTA per row; the row is read twice (second read served by L1/L2).
+// One CTA per row.  Rows of up to 256 * 4 * kRmsVecs floats are read from HBM exactly once and kept in
+// registers between the reduction and the scaling; longer rows are read a second time (from L1/L2).
+constexpr int kRmsVecs = 8;
 __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const float *__restrict__ x,
                                                            const bf16 *__restrict__ gain, int dim, float eps,
                                                            bf16 *__restrict__ out) {
   __shared__ float red[32];
   const float4 *row = reinterpret_cast<const float4 *>(x + (long long)blockIdx.x * dim);
+  const int nvec = dim / 4;
+  const bool cached = nvec <= 256 * kRmsVecs;
+  float4 keep[kRmsVecs];
   float ss = 0.f;
-  for (int v = threadIdx.x; v < dim / 4; v += blockDim.x) {
-    float4 a = row[v];
-    ss += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
+  if (cached) {
+#pragma unroll
+    for (int i = 0; i < kRmsVecs; ++i) {
+      const int v = threadIdx.x + i * 256;
+      keep[i] = (v < nvec) ? __ldcs(row + v) : make_float4(0.f, 0.f, 0.f, 0.f);
+      ss += keep[i].x * keep[i].x + keep[i].y * keep[i].y + keep[i].z * keep[i].z + keep[i].w * keep[i].w;
+    }
+  } else {
+    for (int v = threadIdx.x; v < nvec; v += blockDim.x) {
+      float4 a = row[v];
+      ss += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
+    }
   }
   ss = block_sum(ss, red);
   const float inv = rsqrtf(ss / (float)dim + eps);
-  __nv_bfloat162 *o = reinterpret_cast<__nv_bfloat162 *>(out + (long long)blockIdx.x * dim);
-  const __nv_bfloat162 *g = reinterpret_cast<const __nv_bfloat162 *>(gain);
-  for (int v = threadIdx.x; v < dim / 4; v += blockDim.x) {
-    float4 a = row[v];
-    float2 g0 = __bfloat1622float2(g[2 * v]), g1 = __bfloat1622float2(g[2 * v + 1]);
-    o[2 * v] = __floats2bfloat162_rn(a.x * inv * g0.x, a.y * inv * g0.y);
-    o[2 * v + 1] = __floats2bfloat162_rn(a.z * inv * g1.x, a.w * inv * g1.y);
+  uint2 *o = reinterpret_cast<uint2 *>(out + (long long)blockIdx.x * dim);
+  const uint2 *g = reinterpret_cast<const uint2 *>(gain);
+  auto emit = [&](int v, float4 a) {
+    const uint2 graw = g[v];
+    const float2 g0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&graw.x));
+    const float2 g1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&graw.y));
+    __nv_bfloat162 lo = __floats2bfloat162_rn(a.x * inv * g0.x, a.y * inv * g0.y);
+    __nv_bfloat162 hi = __floats2bfloat162_rn(a.z * inv * g1.x, a.w * inv * g1.y);
+    uint2 packed;
+    packed.x = *reinterpret_cast<uint32_t *>(&lo);
+    packed.y = *reinterpret_cast<uint32_t *>(&hi);
+    o[v] = packed;
+  };
+  if (cached) {
+#pragma unroll
+    for (int i = 0; i < kRmsVecs; ++i) {
+      const int v = threadIdx.x + i * 256;
+      if (v < nvec) emit(v, keep[i]);
+    }
+  } else {
+    for (int v = threadIdx.x; v < nvec; v += blockDim.x) emit(v, row[v]);
   }
 }
 
