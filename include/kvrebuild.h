@@ -244,6 +244,35 @@ int32_t kv_op_paged_attention_noalloc(const float *q_dev, int32_t n_q_heads, con
                                       int32_t layer, const int32_t *block_table_dev, int32_t n_ctx,
                                       float *out_dev, void *stream);
 
+/* ---------------------------------------------------------------- window selection (host scalar code)
+ * The Scheduler Engine's cost model and online selection (Section 4.1, Eqs. 3-9; Section 4.2, Algorithm 1;
+ * Section 4.4, Eq. 10).  Units: seconds, tokens, tokens/s, bytes, bytes/s.  No device work, no allocation. */
+typedef struct {
+  double k_curr;    /* K_curr: current context length (tokens) */
+  double r_p;       /* effective prefill throughput at the target (tokens/s), > 0 */
+  double r_d;       /* per-request decode throughput at the source (tokens/s) */
+  double goodput;   /* B: effective inter-node goodput (bytes/s), > 0 */
+  double s_kv;      /* Eq. (1): KV bytes per token */
+  double t0;        /* T_0: assembly + activation + first decode step (s) */
+  double t_load;    /* T_load: model load latency (0 when resident) */
+  double alpha;     /* weight of T_SIT in Eq. (8), in [0, 1] */
+  double t_remain;  /* predicted remaining time to handover (s) */
+} kv_window_inputs;
+
+typedef struct {
+  double t_w, l_hist, t_hist, t_res, t_sit, t_early, cost;
+} kv_window_eval;
+
+/* Eqs. (3)-(9) for one candidate window T_w. */
+int32_t kv_window_evaluate(const kv_window_inputs *in, double t_w, kv_window_eval *out);
+/* Algorithm 1 after admission: candidates {0, dT, ..., T_limit}, T_limit = min(T_max, T_remain); *best receives the
+ * arg-min (ties: the smallest window), *trigger is 1 iff T_remain <= T_w*. */
+int32_t kv_window_select(const kv_window_inputs *in, double t_max, double d_t, kv_window_eval *best, int32_t *trigger);
+/* Eq. (10): bound on discarded preparation, max{T_max + E_early - T_avail, 0}. */
+double kv_window_waste_bound(double t_max, double e_early, double t_avail);
+/* Telemetry smoothing (Section 4.2): beta * sample + (1 - beta) * old. */
+double kv_ewma(double old_value, double sample, double beta);
+
 /* Event profiler (off by default).  While enabled, every kernel class launched by the operations above is
  * bracketed by CUDA events on the caller's stream.  kv_profile_read waits for the recorded events, adds the
  * elapsed milliseconds and kernel-launch counts per class into the two host arrays (n_kinds >= 14) and clears

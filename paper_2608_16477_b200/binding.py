@@ -20,6 +20,7 @@ EXPORTS = [
     "kv_op_gemm", "kv_op_gemm_reference", "kv_op_rmsnorm",
     "kv_op_attention_prefill", "kv_paged_attention_scratch_bytes", "kv_op_paged_attention", "kv_fill_pattern",
     "kv_profile_enable", "kv_profile_read", "kv_launch_count", "kv_op_paged_attention_noalloc", "kv_check_copy_status", "kv_op_gemv",
+    "kv_window_evaluate", "kv_window_select", "kv_window_waste_bound", "kv_ewma",
 ]
 
 PROFILE_KINDS = ("embed", "rmsnorm", "gemm_qkv", "rope_store", "attention", "gemm_o", "gemm_gate_up", "gemm_down",
@@ -46,6 +47,17 @@ class Weights(C.Structure):
     _fields_ = [("embed_dev", C.c_void_p), ("lm_head_dev", C.c_void_p), ("final_norm_dev", C.c_void_p)] + \
         [(n, C.POINTER(C.c_void_p)) for n in ("attn_norm_dev", "w_qkv_dev", "w_o_dev", "ffn_norm_dev",
                                               "w_gate_up_dev", "w_down_dev")]
+
+
+class WindowInputs(C.Structure):
+    _fields_ = [(n, C.c_double) for n in ("k_curr", "r_p", "r_d", "goodput", "s_kv", "t0", "t_load", "alpha", "t_remain")]
+
+
+class WindowEval(C.Structure):
+    _fields_ = [(n, C.c_double) for n in ("t_w", "l_hist", "t_hist", "t_res", "t_sit", "t_early", "cost")]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_}
 
 
 class CacheDesc(C.Structure):
@@ -96,6 +108,11 @@ def load(build_if_missing: bool = True):
         "kv_fill_pattern": (i32, [vp, i64, C.c_uint64, i64, vp]),
         "kv_op_paged_attention_noalloc": (i32, [vp, i32, C.POINTER(CacheDesc), i32, vp, i32, vp, vp]),
         "kv_check_copy_status": (i32, [vp]),
+        "kv_window_evaluate": (i32, [C.POINTER(WindowInputs), C.c_double, C.POINTER(WindowEval)]),
+        "kv_window_select": (i32, [C.POINTER(WindowInputs), C.c_double, C.c_double, C.POINTER(WindowEval),
+                                   C.POINTER(C.c_int32)]),
+        "kv_window_waste_bound": (C.c_double, [C.c_double, C.c_double, C.c_double]),
+        "kv_ewma": (C.c_double, [C.c_double, C.c_double, C.c_double]),
         "kv_op_gemv": (i32, [vp, vp, i32, i32, i32, vp, C.c_float, vp, vp]),
         "kv_profile_enable": (i32, [i32]),
         "kv_profile_read": (i32, [C.POINTER(C.c_float), C.POINTER(C.c_int64), i32]),
@@ -376,3 +393,24 @@ def kv_op_gemv(w, x, mode: int, y, gain=None, eps: float = 0.0, stream=None, n=N
     rows, k = w.shape
     n = n if n is not None else (rows // 2 if mode == 2 else rows)
     _check(load().kv_op_gemv(_ptr(w), _ptr(x), n, k, mode, _ptr(gain), eps, _ptr(y), _stream(stream)), "kv_op_gemv")
+
+
+def kv_window_evaluate(t_w: float, **inputs) -> dict:
+    win, out = WindowInputs(**inputs), WindowEval()
+    _check(load().kv_window_evaluate(C.byref(win), t_w, C.byref(out)), "kv_window_evaluate")
+    return out.as_dict()
+
+
+def kv_window_select(t_max: float, d_t: float, **inputs):
+    """Returns (evaluation at T_w*, trigger)."""
+    win, out, trig = WindowInputs(**inputs), WindowEval(), C.c_int32()
+    _check(load().kv_window_select(C.byref(win), t_max, d_t, C.byref(out), C.byref(trig)), "kv_window_select")
+    return out.as_dict(), bool(trig.value)
+
+
+def kv_window_waste_bound(t_max: float, e_early: float, t_avail: float) -> float:
+    return float(load().kv_window_waste_bound(t_max, e_early, t_avail))
+
+
+def kv_ewma(old: float, sample: float, beta: float) -> float:
+    return float(load().kv_ewma(old, sample, beta))
