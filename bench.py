@@ -46,7 +46,7 @@ WORKLOADS = {
 
 # DRAM bytes (read + write) of one gate/up GEMM launch at the 32b-4k workload, from the ncu capture
 # summarised under profiles/ (same shape as the bench's launch: M 4096, K 5120, 2 x 25600 weight rows).
-NCU_TRAFFIC_BYTES = {"32b-4k": 870.5e6}   # profiles/gemm_tc_gate_up_32b-4k.md: 665.8 MB read + 204.7 MB written
+NCU_TRAFFIC_BYTES = {"32b-4k": 857.2e6}   # profiles/gemm_tc_gate_up_32b-4k.md: 653.7 MB read + 203.5 MB written
 
 
 def peaks():
