@@ -37,6 +37,14 @@ constexpr float kRescaleThreshold = 8.0f;
 constexpr int kRegsOther = 72;      // registers per thread of warps 0-3 after the hand-back
 constexpr int kRegsSoftmax = 216;   // registers per thread of the softmax warps
 
+#ifdef KV_ATTN_TRACE
+__device__ long long g_attn_trace[64 * 16];
+#define KV_ATRACE(slot, idx) \
+  do { if (blockIdx.x == 0 && (idx) < 64) g_attn_trace[(idx) * 16 + (slot)] = clock64(); } while (0)
+#else
+#define KV_ATRACE(slot, idx) do { } while (0)
+#endif
+
 enum AttnTag { ATAG_Q = 11, ATAG_KV_EMPTY = 12, ATAG_K = 13, ATAG_V = 14, ATAG_S = 15, ATAG_P = 16, ATAG_O = 17 };
 
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
@@ -198,6 +206,7 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
           ok = tc::mbar_wait(bar(B_P, t), j & 1, abort_flag, status, ATAG_P) &&
                tc::mbar_wait(bar(B_V, st), ph, abort_flag, status, ATAG_V);
           if (!ok) break;
+          KV_ATRACE(8 + t * 2, j);
           tc::tc_fence_after();
 #pragma unroll
           for (int ks = 0; ks < kBN / 16; ++ks)   // 16 keys per slice: 8 TMEM columns of P, 2048 bytes of V
@@ -212,6 +221,7 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
           } else {
             tc::umma_commit(bar(B_O, t));
           }
+          KV_ATRACE(9 + t * 2, j);
         }
       }
     }
@@ -233,6 +243,7 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
       ok = tc::mbar_wait(bar(B_S, t), j & 1, abort_flag, status, ATAG_S);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
+      if (quarter == 0 && lane == 0) KV_ATRACE(t * 4 + 0, j);
       tc::tc_fence_after();
       const bool diag = (j * kBN + kBN - 1 > pos0 + m0);   // tile reaches past the first row's position
       const int limit = qi - j * kBN;              // keys with column > limit are masked
@@ -243,6 +254,7 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
       tc::tmem_ld32(s_t + 64, r2);
       tc::tmem_ld32(s_t + 96, r3);
       tc::tmem_ld_wait();
+      if (quarter == 0 && lane == 0) KV_ATRACE(t * 4 + 1, j);
       float mx = -INFINITY;
       if (!diag) {
 #pragma unroll
@@ -284,6 +296,7 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
           tmem_st32(o_t + c * 32, r);
         }
       }
+      if (quarter == 0 && lane == 0) KV_ATRACE(t * 4 + 2, j);
       // probabilities, written over S as packed bf16 (two keys per 32-bit column); masked scores are -inf -> 0
       const float neg_m = -m_ref;
       float sum0 = 0.f, sum1 = 0.f;
@@ -307,6 +320,7 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
       tc::tmem_st_wait();
       tc::tc_fence_before();
       tc::mbar_arrive(bar(B_P, t));
+      if (quarter == 0 && lane == 0) KV_ATRACE(t * 4 + 3, j);
     }
     if (ok) {
       ok = tc::mbar_wait(bar(B_O, t), 0, abort_flag, status, ATAG_O);
@@ -418,5 +432,11 @@ int attention_prefill_tc(const bf16 *qkv_ctx, int n_tokens, int pos0, int n_q_he
   KV_CUDA(cudaGetLastError());
   return KV_OK;
 }
+
+#ifdef KV_ATTN_TRACE
+extern "C" int kv_debug_attn_trace(long long *out_host) {
+  return cudaMemcpyFromSymbol(out_host, g_attn_trace, sizeof(long long) * 64 * 16) == cudaSuccess ? 0 : -13;
+}
+#endif
 
 }  // namespace kvr
