@@ -114,14 +114,14 @@ def run_reference(args):
     shape = synth.SHAPES[shape_name]
     sample_tokens = min(prefix, args.ref_tokens)
     run = oracle_sample(shape, sample_tokens)
-    for _ in range(args.ref_warmup):
+    for _ in range(max(args.ref_warmup, args.warmup if args.warmup_given else 0)):
         run()
     times = [run() for _ in range(args.steps)]
     secs = sum(times) / len(times)
     value = sample_tokens / (secs * shape.n_layers)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.ref_warmup, "ms_per_step": secs * 1e3, "higher_is_better": True,
+        "steps": args.steps, "warmup": max(args.ref_warmup, args.warmup if args.warmup_given else 0), "ms_per_step": secs * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": args.workload, "prefix_tokens": prefix, "suffix_tokens": suffix,
                    "step": f"one decoder layer of {shape.n_layers} over {sample_tokens} prefix tokens (bounded sample)"},
@@ -394,18 +394,93 @@ def run_ours(args):
     return 0
 
 
+# ------------------------------------------------------------------------------------------ pack/unpack stress
+def stress_geometry(kv, torch, shape):
+    """Source pool of 32,768 blocks (128 GiB at the 32B shape) when it fits beside a 5,120-block destination pool
+    and the 18.1 GiB of wire buffers; otherwise the source pool is halved until it does (only referenced pages
+    are touched, so the pool size changes the address spread, not the bytes moved)."""
+    counts = list(synth.STRESS_BLOCK_COUNTS)
+    total = sum(counts)
+    page = synth.kv_page_bytes(shape)
+    block_bytes = 2 * shape.n_layers * page
+    dst_blocks = 5120
+    free, _ = torch.cuda.mem_get_info()
+    src_blocks = 32768
+    while src_blocks > total and (src_blocks + dst_blocks + total) * block_bytes + (2 << 30) > free:
+        src_blocks //= 2
+    return counts, total, src_blocks, dst_blocks, block_bytes
+
+
+def run_pack_stress(args):
+    import torch
+    import paper_2608_16477_b200 as kv
+    kv.load()
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    shape = synth.SHAPES["32b"]
+    counts, total, src_blocks, dst_blocks, block_bytes = stress_geometry(kv, torch, shape)
+    src = kv.PagedCache(shape, src_blocks)
+    dst = kv.PagedCache(shape, dst_blocks, fill=0)
+    kv.kv_fill_pattern(src.data, src.data.numel() * 2, seed=77)
+    offs = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+    src_ids = synth.block_permutation(1, src_blocks)[:total]
+    dst_ids = synth.block_permutation(2, dst_blocks)[:total]
+    wires = [torch.empty(c * block_bytes, dtype=torch.uint8, device="cuda") for c in counts]
+    stream = torch.cuda.current_stream()
+
+    def timed(fn, reps):
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+    pack = lambda: kv.kv_pack_blocks_batched(src, offs, src_ids, wires)
+    unpack = lambda: kv.kv_unpack_blocks_batched(dst, offs, dst_ids, wires)
+    for _ in range(max(args.warmup, 3)):
+        pack(); unpack()
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    l0 = kv.kv_launch_count()
+    pack_ms = timed(pack, args.steps)
+    unpack_ms = timed(unpack, args.steps)
+    launches = kv.kv_launch_count() - l0
+    clocks = sampler.stop()
+    kv.kv_check_copy_status()
+    pk = peaks()
+    payload = total * block_bytes
+    gbs = lambda ms: 2 * payload / (ms * 1e-3) / 1e9
+    line = {"metric": "kv_pack_unpack_gbs", "value": gbs(pack_ms), "unit": "GB/s", "n_gpus": 1, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": pack_ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+            "config": {"workload": "pack-stress", "requests": len(counts), "blocks": total, "payload_bytes": payload,
+                       "src_pool_blocks": src_blocks, "dst_pool_blocks": dst_blocks,
+                       "l2": "inputs larger than L2 (18.1 GiB payload per launch set)"},
+            "clocks": clocks, "gpu_launches": int(launches),
+            "roofline": {"bound": "hbm", "kernel": "copy_pages_kernel", "achieved": gbs(pack_ms), "peak": pk["hbm_gbs"],
+                         "unit": "GB/s", "frac": gbs(pack_ms) / pk["hbm_gbs"], "peak_source": pk["source"], "traffic": None},
+            "pack": {"gbs": gbs(pack_ms), "ms": pack_ms, "frac_of_hbm": gbs(pack_ms) / pk["hbm_gbs"]},
+            "unpack": {"gbs": gbs(unpack_ms), "ms": unpack_ms, "frac_of_hbm": gbs(unpack_ms) / pk["hbm_gbs"]}}
+    print(json.dumps(line))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="32b-4k", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="32b-4k", choices=sorted(WORKLOADS) + ["pack-stress"])
     ap.add_argument("--layers", type=int, default=0, help="debug: reduced depth (invalid as a bench number)")
     ap.add_argument("--ref-tokens", type=int, default=2048, help="prefix tokens in the oracle's bounded sample")
     ap.add_argument("--ref-warmup", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    args.warmup_given = any(a == "--warmup" or a.startswith("--warmup=") for a in sys.argv[1:])
+    if args.workload == "pack-stress" and args.impl != "reference":
+        return run_pack_stress(args)
     if args.impl == "reference":
         return run_reference(args)
     return run_ours(args)

@@ -147,3 +147,37 @@ def test_8b_full_depth_against_oracle(kv):
         bound = BF16_FLOOR if l == 0 else PER_LAYER_NOISE * np.sqrt(l)
         assert ek <= bound and ev <= bound, (l, ek, ev, bound)
     assert lg["rel_l2"] <= PER_LAYER_NOISE * np.sqrt(s.n_layers), lg
+
+
+def test_pack_unpack_stress_16_requests_full_size(kv):
+    """The 16-request stress workload at full size: 4,639 blocks (18.1 GiB) gathered from a source pool of up to
+    32,768 blocks into per-request wire buffers and scattered into a second cache, in the batched launch form.
+    Sampled pages are checked against the host-generated counter pattern (what the oracle's pack would copy)."""
+    import torch
+    from bench import stress_geometry
+    s = synth.SHAPES["32b"]
+    counts, total, src_blocks, dst_blocks, block_bytes = stress_geometry(kv, torch, s)
+    assert total == 4639 and total * block_bytes == 4639 * 4 * 1024 * 1024
+    page = synth.kv_page_bytes(s)
+    src = kv.PagedCache(s, src_blocks)
+    dst = kv.PagedCache(s, dst_blocks, fill=0)
+    kv.kv_fill_pattern(src.data, src.data.numel() * 2, seed=77)
+    offs = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+    src_ids = synth.block_permutation(1, src_blocks)[:total]
+    dst_ids = synth.block_permutation(2, dst_blocks)[:total]
+    wires = [torch.empty(c * block_bytes, dtype=torch.uint8, device="cuda") for c in counts]
+    kv.kv_pack_blocks_batched(src, offs, src_ids, wires)
+    kv.kv_unpack_blocks_batched(dst, offs, dst_ids, wires)
+    kv.kv_check_copy_status()
+    rng = np.random.default_rng(9)
+    for _ in range(96):
+        r = int(rng.integers(0, len(counts))); i = int(rng.integers(0, counts[r]))
+        l = int(rng.integers(0, s.n_layers)); kvi = int(rng.integers(0, 2))
+        b_src, b_dst = int(src_ids[offs[r] + i]), int(dst_ids[offs[r] + i])
+        want = synth.pattern_bytes(77, ((l * 2 + kvi) * src_blocks + b_src) * page, page)
+        w_off = ((i * s.n_layers + l) * 2 + kvi) * page
+        assert np.array_equal(wires[r][w_off:w_off + page].cpu().numpy(), want)
+        assert np.array_equal(dst.data[l, kvi, b_dst].cpu().numpy().view(np.uint8), want)
+    unused = np.setdiff1d(np.arange(dst_blocks), dst_ids)
+    assert not dst.data[:, :, torch.from_numpy(unused).cuda()].any()
+    print("stress geometry:", dict(src_blocks=src_blocks, dst_blocks=dst_blocks, blocks=total))
