@@ -142,6 +142,18 @@ int32_t kv_prefill_prefix(kv_model *m, const kv_cache_desc *cache,
                           void *workspace_dev, int64_t workspace_bytes,
                           float *logits_out_dev, void *stream);
 
+/* Several prefix reconstructions in one call (concurrent migrations sharing the target GPU, Section 4.5:
+ * handover-handover contention).  Request r owns tokens token_ids_host[token_offsets_host[r] ..
+ * token_offsets_host[r+1]) and the block table block_tables_host[table_offsets_host[r] .. table_offsets_host[r+1]);
+ * every request starts at position 0.  All rows go through the projections together (one GEMM per layer over
+ * the sum of the prefix lengths), attention runs per request.  Physical blocks must be distinct across the whole
+ * batch.  Results are identical to n_req separate kv_prefill_prefix calls.  workspace: kv_workspace_bytes(m,
+ * KV_OP_PREFILL, total tokens).  logits_out_dev: NULL or fp32 [n_req, vocab]. */
+int32_t kv_prefill_prefix_batched(kv_model *m, const kv_cache_desc *cache, int32_t n_req,
+                                  const int32_t *token_offsets_host, const int32_t *token_ids_host,
+                                  const int32_t *table_offsets_host, const int32_t *block_tables_host,
+                                  void *workspace_dev, int64_t workspace_bytes, float *logits_out_dev, void *stream);
+
 /* Source-side suffix block extraction (Section 5: physical block ids from the block manager ->
  * per-layer KV tensors -> bytes).  wire[i] <- all pages of block block_ids_host[i], i in logical
  * order.  Bytes are copied verbatim.  Duplicate ids are allowed. */

@@ -5,7 +5,7 @@ Every step of the path runs in the library's CUDA kernels; this package only mar
 shared library is missing and cannot be built.
 """
 from .binding import (KVError, load, lib_path, status_string, Model, PagedCache, kv_bytes_per_token,
-                      kv_prefill_prefix, kv_pack_blocks, kv_unpack_assemble, kv_decode_step,
+                      kv_prefill_prefix, kv_prefill_prefix_batched, kv_pack_blocks, kv_unpack_assemble, kv_decode_step,
                       kv_pack_blocks_batched, kv_unpack_blocks_batched, kv_workspace_bytes,
                       kv_check_device_status, kv_check_copy_status, kv_window_evaluate, kv_window_select,
                       kv_window_waste_bound, kv_ewma, kv_op_gemm, kv_op_gemm_reference, kv_op_gemv, kv_op_rmsnorm,

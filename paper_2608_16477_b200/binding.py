@@ -20,7 +20,7 @@ EXPORTS = [
     "kv_op_gemm", "kv_op_gemm_reference", "kv_op_rmsnorm",
     "kv_op_attention_prefill", "kv_paged_attention_scratch_bytes", "kv_op_paged_attention", "kv_fill_pattern",
     "kv_profile_enable", "kv_profile_read", "kv_launch_count", "kv_op_paged_attention_noalloc", "kv_check_copy_status", "kv_op_gemv",
-    "kv_window_evaluate", "kv_window_select", "kv_window_waste_bound", "kv_ewma",
+    "kv_window_evaluate", "kv_window_select", "kv_window_waste_bound", "kv_ewma", "kv_prefill_prefix_batched",
 ]
 
 PROFILE_KINDS = ("embed", "rmsnorm", "gemm_qkv", "rope_store", "attention", "gemm_o", "gemm_gate_up", "gemm_down",
@@ -93,6 +93,7 @@ def load(build_if_missing: bool = True):
         "kv_bytes_per_token": (i64, [i32, i32, i32, i32]),
         "kv_check_device_status": (i32, [vp, vp]),
         "kv_prefill_prefix": (i32, [vp, C.POINTER(CacheDesc), pi32, i32, i32, pi32, i32, vp, i64, vp, vp]),
+        "kv_prefill_prefix_batched": (i32, [vp, C.POINTER(CacheDesc), i32, pi32, pi32, pi32, pi32, vp, i64, vp, vp]),
         "kv_pack_blocks": (i32, [C.POINTER(CacheDesc), pi32, i32, vp, i64, i32, vp]),
         "kv_unpack_assemble": (i32, [C.POINTER(CacheDesc), vp, i64, i32, pi32, pi32, i32, pi32, i32, i32,
                                      C.c_uint32, C.c_uint32, pi32, vp]),
@@ -414,3 +415,19 @@ def kv_window_waste_bound(t_max: float, e_early: float, t_avail: float) -> float
 
 def kv_ewma(old: float, sample: float, beta: float) -> float:
     return float(load().kv_ewma(old, sample, beta))
+
+
+def kv_prefill_prefix_batched(model: Model, cache: PagedCache, token_id_lists, block_tables, logits_out=None,
+                              workspace=None, stream=None):
+    """Prefix reconstruction of several requests in one call (lists of per-request token ids / block tables)."""
+    tok_off = np.concatenate([[0], np.cumsum([len(t) for t in token_id_lists])]).astype(np.int32)
+    tab_off = np.concatenate([[0], np.cumsum([len(t) for t in block_tables])]).astype(np.int32)
+    ids, pids = _i32(np.concatenate([np.asarray(t, dtype=np.int32) for t in token_id_lists]))
+    tabs, ptabs = _i32(np.concatenate([np.asarray(t, dtype=np.int32) for t in block_tables]))
+    toff, ptoff = _i32(tok_off)
+    boff, pboff = _i32(tab_off)
+    ws = workspace if workspace is not None else model.workspace(KV_OP_PREFILL, int(tok_off[-1]))
+    _check(load().kv_prefill_prefix_batched(model.handle, C.byref(cache.desc), len(token_id_lists), ptoff, pids, pboff,
+                                            ptabs, _ptr(ws), ws.numel(), _ptr(logits_out), _stream(stream)),
+           "kv_prefill_prefix_batched")
+    return ws

@@ -139,7 +139,7 @@ struct Carver {
 
 struct PrefillWs {
   DeviceStatus *status;
-  int *ids, *table;
+  int *ids, *table, *row_meta;
   float2 *rope;
   float *x, *xf;
   bf16 *h, *qkv, *attn, *mid;
@@ -154,6 +154,7 @@ PrefillWs carve_prefill(const kv_model_desc &d, void *base, int max_tokens, int 
   w.status = c.take<DeviceStatus>(1);
   w.ids = c.take<int>(t);
   w.table = c.take<int>((t + block_size - 1) / block_size + 1);
+  w.row_meta = c.take<int>(2 * t);
   w.rope = c.take<float2>(t * (d.head_dim / 2));
   w.x = c.take<float>(t * d.hidden);
   w.xf = c.take<float>(d.hidden);
@@ -321,6 +322,85 @@ int32_t kv_check_device_status(const void *workspace_dev, void *stream) {
   return KV_OK;
 }
 
+#define KV_TRY(expr)            \
+  do {                          \
+    int rc__ = (expr);          \
+    if (rc__ != KV_OK) return rc__; \
+  } while (0)
+
+namespace {
+
+// One request inside a prefill launch sequence: rows [row0, row0 + n_tokens) of the activation buffers.
+struct PrefillSegment {
+  int row0, n_tokens;
+  float *logits;   // nullable
+};
+
+// The layer loop shared by the single-request and the batched entry points.  All rows of all segments go
+// through the projections together; attention runs per segment (requests do not attend to each other).
+// Single request: pos0 may be > 0 (continued prefill) and rows map to the request's block table.  Batched:
+// pos0 = 0 and every row carries its own position and physical block (row_pos / row_block on the device).
+int prefill_layers(kv_model *m, const CacheView &cv, PrefillWs &w, int total_rows, int pos0,
+                   const std::vector<PrefillSegment> &segs, const int *row_pos, const int *row_block, bool any_logits,
+                   cudaStream_t st) {
+  const kv_model_desc &d = m->d;
+  const int t = total_rows;
+  const int qkv_dim = (d.n_q_heads + 2 * d.n_kv_heads) * d.head_dim;
+  const int q_dim = d.n_q_heads * d.head_dim;
+  { ProfScope ps(PROF_ROPE_STORE, st); KV_TRY(rope_table(w.rope, pos0, t, d.head_dim, d.rope_base, st, row_pos)); }
+  // the qkv buffer has one row per context position; the chunk's rows start at pos0
+  const bool tc_attention = attention_tc_supported(d.n_q_heads, d.n_kv_heads, d.head_dim);
+  bf16 *qkv_chunk = w.qkv + (long long)pos0 * qkv_dim;
+  { ProfScope ps(PROF_EMBED, st); KV_TRY(embed_rows(m->embed, w.ids, t, d.hidden, w.x, st)); }
+  for (int l = 0; l < d.n_layers; ++l) {
+    { ProfScope ps(PROF_RMSNORM, st); KV_TRY(rmsnorm_rows(w.x, m->attn_norm[l], t, d.hidden, d.rms_eps, w.h, st)); }
+    {
+      ProfScope ps(PROF_GEMM_QKV, st);
+      QkvRopeArgs qa;
+      qa.rope = w.rope;
+      qa.block_table = w.table;
+      qa.row_pos = row_pos;
+      qa.row_block = row_block;
+      qa.cache = cv;
+      qa.pos0 = pos0;
+      qa.head_dim = d.head_dim;
+      qa.n_q_heads = d.n_q_heads;
+      qa.n_kv_heads = d.n_kv_heads;
+      qa.layer = l;
+      KV_TRY(run_gemm(m, w.h, d.hidden, m->w_qkv[l], t, qkv_dim, d.hidden, GEMM_QKV_ROPE, qkv_chunk, nullptr, w.status, st, &qa));
+    }
+    if (l == d.n_layers - 1 && !any_logits) break;   // K/V of the last layer are complete
+    {
+      ProfScope ps(PROF_ATTENTION, st);
+      for (const PrefillSegment &sg : segs) {
+        bf16 *seg_qkv = w.qkv + (long long)sg.row0 * qkv_dim;     // rows of this request (its context starts here)
+        bf16 *seg_out = w.attn + (long long)sg.row0 * q_dim;
+        if (tc_attention) {
+          KV_TRY(gather_prefix_kv(seg_qkv, pos0, d.n_q_heads, d.n_kv_heads, d.head_dim, cv, l, w.table, st));
+          KV_TRY(attention_prefill_tc(seg_qkv, sg.n_tokens, pos0, d.n_q_heads, d.n_kv_heads, d.head_dim, seg_out,
+                                      reinterpret_cast<int *>(w.status), st));
+        } else {
+          KV_TRY(attention_prefill(seg_qkv + (long long)pos0 * qkv_dim, sg.n_tokens, pos0, d.n_q_heads, d.n_kv_heads,
+                                   d.head_dim, cv, l, w.table, seg_out, reinterpret_cast<int *>(w.status), st));
+        }
+      }
+    }
+    { ProfScope ps(PROF_GEMM_O, st); KV_TRY(run_gemm(m, w.attn, q_dim, m->w_o[l], t, d.hidden, q_dim, GEMM_RESID_F32, nullptr, w.x, w.status, st)); }
+    { ProfScope ps(PROF_RMSNORM, st); KV_TRY(rmsnorm_rows(w.x, m->ffn_norm[l], t, d.hidden, d.rms_eps, w.h, st)); }
+    { ProfScope ps(PROF_GEMM_GATE_UP, st); KV_TRY(run_gemm(m, w.h, d.hidden, m->w_gate_up[l], t, d.ffn, d.hidden, GEMM_SWIGLU, w.mid, nullptr, w.status, st)); }
+    { ProfScope ps(PROF_GEMM_DOWN, st); KV_TRY(run_gemm(m, w.mid, d.ffn, m->w_down[l], t, d.hidden, d.ffn, GEMM_RESID_F32, nullptr, w.x, w.status, st)); }
+  }
+  for (const PrefillSegment &sg : segs) {
+    if (sg.logits == nullptr) continue;
+    ProfScope ps(PROF_LM_HEAD, st);
+    KV_TRY(gemv(m->lm_head, w.x + (long long)(sg.row0 + sg.n_tokens - 1) * d.hidden, d.vocab, d.hidden, 0, sg.logits, st,
+                m->final_norm, d.rms_eps));
+  }
+  return KV_OK;
+}
+
+}  // namespace
+
 int32_t kv_prefill_prefix(kv_model *m, const kv_cache_desc *cache, const int32_t *token_ids_host, int32_t n_tokens,
                           int32_t pos0, const int32_t *block_table_host, int32_t n_blocks, void *workspace_dev,
                           int64_t workspace_bytes, float *logits_out_dev, void *stream) {
@@ -344,62 +424,56 @@ int32_t kv_prefill_prefix(kv_model *m, const kv_cache_desc *cache, const int32_t
   if (workspace_bytes < w.bytes) return KV_ERR_WORKSPACE;
   // buffers are sized by the context length n_ctx; only the first n_tokens rows are used
   cudaStream_t st = (cudaStream_t)stream;
-  const CacheView cv = make_view(cache);
-  const int t = n_tokens;
-  const int qkv_dim = (d.n_q_heads + 2 * d.n_kv_heads) * d.head_dim;
-  const int q_dim = d.n_q_heads * d.head_dim;
-
   KV_CUDA(cudaMemsetAsync(w.status, 0, sizeof(DeviceStatus), st));
-  KV_CUDA(cudaMemcpyAsync(w.ids, token_ids_host, sizeof(int) * t, cudaMemcpyHostToDevice, st));
+  KV_CUDA(cudaMemcpyAsync(w.ids, token_ids_host, sizeof(int) * n_tokens, cudaMemcpyHostToDevice, st));
   KV_CUDA(cudaMemcpyAsync(w.table, block_table_host, sizeof(int) * need_blocks, cudaMemcpyHostToDevice, st));
-#define KV_TRY(expr)            \
-  do {                          \
-    int rc__ = (expr);          \
-    if (rc__ != KV_OK) return rc__; \
-  } while (0)
-  { ProfScope ps(PROF_ROPE_STORE, st); KV_TRY(rope_table(w.rope, pos0, t, d.head_dim, d.rope_base, st)); }
-  // the qkv buffer has one row per context position; the chunk's rows start at pos0
-  const bool tc_attention = attention_tc_supported(d.n_q_heads, d.n_kv_heads, d.head_dim);
-  bf16 *qkv_chunk = w.qkv + (long long)pos0 * qkv_dim;
-  { ProfScope ps(PROF_EMBED, st); KV_TRY(embed_rows(m->embed, w.ids, t, d.hidden, w.x, st)); }
-  for (int l = 0; l < d.n_layers; ++l) {
-    { ProfScope ps(PROF_RMSNORM, st); KV_TRY(rmsnorm_rows(w.x, m->attn_norm[l], t, d.hidden, d.rms_eps, w.h, st)); }
-    {
-      ProfScope ps(PROF_GEMM_QKV, st);
-      QkvRopeArgs qa;
-      qa.rope = w.rope;
-      qa.block_table = w.table;
-      qa.cache = cv;
-      qa.pos0 = pos0;
-      qa.head_dim = d.head_dim;
-      qa.n_q_heads = d.n_q_heads;
-      qa.n_kv_heads = d.n_kv_heads;
-      qa.layer = l;
-      KV_TRY(run_gemm(m, w.h, d.hidden, m->w_qkv[l], t, qkv_dim, d.hidden, GEMM_QKV_ROPE, qkv_chunk, nullptr, w.status, st, &qa));
+  std::vector<PrefillSegment> segs{{0, n_tokens, logits_out_dev}};
+  return prefill_layers(m, make_view(cache), w, n_tokens, pos0, segs, nullptr, nullptr, logits_out_dev != nullptr, st);
+}
+
+int32_t kv_prefill_prefix_batched(kv_model *m, const kv_cache_desc *cache, int32_t n_req,
+                                  const int32_t *token_offsets_host, const int32_t *token_ids_host,
+                                  const int32_t *table_offsets_host, const int32_t *block_tables_host,
+                                  void *workspace_dev, int64_t workspace_bytes, float *logits_out_dev, void *stream) {
+  if (m == nullptr || n_req <= 0 || token_offsets_host == nullptr || token_ids_host == nullptr ||
+      table_offsets_host == nullptr || block_tables_host == nullptr)
+    return KV_ERR_ARG;
+  const kv_model_desc &d = m->d;
+  int rc = check_cache_vs_model(cache, d);
+  if (rc != KV_OK) return rc;
+  const int bs = cache->block_size;
+  if (token_offsets_host[0] != 0 || table_offsets_host[0] != 0) return KV_ERR_ARG;
+  const int total = token_offsets_host[n_req];
+  const int total_blocks = table_offsets_host[n_req];
+  if (total <= 0 || total_blocks <= 0) return KV_ERR_ARG;
+  std::vector<int> row_meta(2 * (size_t)total);   // [0, total): position in request, [total, 2 total): physical block
+  std::vector<PrefillSegment> segs;
+  for (int r = 0; r < n_req; ++r) {
+    const int n_tok = token_offsets_host[r + 1] - token_offsets_host[r];
+    const int n_blk = table_offsets_host[r + 1] - table_offsets_host[r];
+    if (n_tok <= 0 || n_blk < 0) return KV_ERR_ARG;
+    if ((long long)n_blk * bs < n_tok) return KV_ERR_TABLE_SHORT;
+    const int32_t *tab = block_tables_host + table_offsets_host[r];
+    for (int i = 0; i < n_tok; ++i) {
+      row_meta[token_offsets_host[r] + i] = i;
+      row_meta[(size_t)total + token_offsets_host[r] + i] = tab[i / bs];
     }
-    if (l == d.n_layers - 1 && logits_out_dev == nullptr) break;   // K/V of the last layer are complete
-    {
-      ProfScope ps(PROF_ATTENTION, st);
-      if (tc_attention) {
-        KV_TRY(gather_prefix_kv(w.qkv, pos0, d.n_q_heads, d.n_kv_heads, d.head_dim, cv, l, w.table, st));
-        KV_TRY(attention_prefill_tc(w.qkv, t, pos0, d.n_q_heads, d.n_kv_heads, d.head_dim, w.attn,
-                                    reinterpret_cast<int *>(w.status), st));
-      } else {
-        KV_TRY(attention_prefill(qkv_chunk, t, pos0, d.n_q_heads, d.n_kv_heads, d.head_dim, cv, l, w.table, w.attn,
-                                 reinterpret_cast<int *>(w.status), st));
-      }
-    }
-    { ProfScope ps(PROF_GEMM_O, st); KV_TRY(run_gemm(m, w.attn, q_dim, m->w_o[l], t, d.hidden, q_dim, GEMM_RESID_F32, nullptr, w.x, w.status, st)); }
-    { ProfScope ps(PROF_RMSNORM, st); KV_TRY(rmsnorm_rows(w.x, m->ffn_norm[l], t, d.hidden, d.rms_eps, w.h, st)); }
-    { ProfScope ps(PROF_GEMM_GATE_UP, st); KV_TRY(run_gemm(m, w.h, d.hidden, m->w_gate_up[l], t, d.ffn, d.hidden, GEMM_SWIGLU, w.mid, nullptr, w.status, st)); }
-    { ProfScope ps(PROF_GEMM_DOWN, st); KV_TRY(run_gemm(m, w.mid, d.ffn, m->w_down[l], t, d.hidden, d.ffn, GEMM_RESID_F32, nullptr, w.x, w.status, st)); }
+    segs.push_back({token_offsets_host[r], n_tok, logits_out_dev ? logits_out_dev + (long long)r * d.vocab : nullptr});
   }
-  if (logits_out_dev != nullptr) {
-    ProfScope ps(PROF_LM_HEAD, st);
-    KV_TRY(gemv(m->lm_head, w.x + (long long)(t - 1) * d.hidden, d.vocab, d.hidden, 0, logits_out_dev, st,
-                m->final_norm, d.rms_eps));
-  }
-  return KV_OK;
+  // physical blocks: in range and distinct across ALL requests (two requests must never share a page)
+  rc = check_ids(block_tables_host, total_blocks, cache->num_blocks, true);
+  if (rc != KV_OK) return rc;
+  for (int i = 0; i < total; ++i)
+    if (token_ids_host[i] < 0 || token_ids_host[i] >= d.vocab) return KV_ERR_TOKEN_RANGE;
+  if (workspace_dev == nullptr || ((uintptr_t)workspace_dev & 1023)) return KV_ERR_WORKSPACE;
+  PrefillWs w = carve_prefill(d, workspace_dev, total, bs);
+  if (workspace_bytes < w.bytes) return KV_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  KV_CUDA(cudaMemsetAsync(w.status, 0, sizeof(DeviceStatus), st));
+  KV_CUDA(cudaMemcpyAsync(w.ids, token_ids_host, sizeof(int) * total, cudaMemcpyHostToDevice, st));
+  KV_CUDA(cudaMemcpyAsync(w.row_meta, row_meta.data(), sizeof(int) * 2 * total, cudaMemcpyHostToDevice, st));
+  return prefill_layers(m, make_view(cache), w, total, 0, segs, w.row_meta, w.row_meta + total, logits_out_dev != nullptr,
+                        st);
 }
 
 int32_t kv_decode_step(kv_model *m, const kv_cache_desc *cache, int32_t token_id, int32_t pos,

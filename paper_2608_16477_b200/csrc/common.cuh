@@ -66,8 +66,10 @@ enum GemmMode { GEMM_STORE_BF16 = 0, GEMM_RESID_F32 = 1, GEMM_SWIGLU = 2, GEMM_Q
 
 // Extra arguments of the fused QKV epilogue: RoPE on the accumulators, K/V stored into the paged cache.
 struct QkvRopeArgs {
-  const float2 *rope;       // [n_tokens, head_dim/2] (cos, sin) of positions pos0 .. pos0+n_tokens-1
-  const int *block_table;   // device
+  const float2 *rope;       // [n_tokens, head_dim/2] (cos, sin) of each row's position
+  const int *block_table;   // device; single request: row r is position pos0 + r of this table
+  const int *row_pos;       // batched requests (else nullptr): position of each row inside its request
+  const int *row_block;     // batched requests: physical block that holds each row
   CacheView cache;
   int pos0, head_dim, n_q_heads, n_kv_heads, layer;
 };
@@ -79,7 +81,9 @@ int gemm_simt(const bf16 *a, int lda, const bf16 *w, int m, int n, int k, int mo
 
 int embed_rows(const bf16 *embed, const int *ids_dev, int n_tokens, int hidden, float *x, cudaStream_t st);
 int rmsnorm_rows(const float *x, const bf16 *gain, int rows, int dim, float eps, bf16 *out, cudaStream_t st);
-int rope_table(float2 *table, int pos0, int n_tokens, int head_dim, float base, cudaStream_t st);
+// positions pos0 + t, or row_pos[t] when row_pos is given (rows of several requests)
+int rope_table(float2 *table, int pos0, int n_tokens, int head_dim, float base, cudaStream_t st,
+               const int *row_pos = nullptr);
 inline bool attention_tc_supported(int n_q_heads, int n_kv_heads, int head_dim) {
   return (head_dim == 64 || head_dim == 128) && ((n_q_heads / n_kv_heads) % 2 == 0);
 }

@@ -106,20 +106,22 @@ int rmsnorm_rows(const float *x, const bf16 *gain, int rows, int dim, float eps,
 
 // table[t, j] = (cos, sin)(pos * base^(-2j/d)), angle formed in fp64 so that positions in the
 // tens of thousands keep full fp32 accuracy after the final rounding.
-__global__ void rope_table_kernel(float2 *table, int pos0, int n_tokens, int half, float base) {
+__global__ void rope_table_kernel(float2 *table, int pos0, int n_tokens, int half, float base,
+                                  const int *__restrict__ row_pos) {
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= n_tokens * half) return;
   const int t = idx / half, j = idx - t * half;
   const double theta = pow((double)base, -(double)j / (double)half);
   double s, c;
-  sincos((double)(pos0 + t) * theta, &s, &c);
+  const int pos = row_pos != nullptr ? row_pos[t] : pos0 + t;
+  sincos((double)pos * theta, &s, &c);
   table[idx] = make_float2((float)c, (float)s);
 }
 
-int rope_table(float2 *table, int pos0, int n_tokens, int head_dim, float base, cudaStream_t st) {
+int rope_table(float2 *table, int pos0, int n_tokens, int head_dim, float base, cudaStream_t st, const int *row_pos) {
   const int n = n_tokens * (head_dim / 2);
   if (n <= 0) return KV_OK;
-  rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(table, pos0, n_tokens, head_dim / 2, base);
+  rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(table, pos0, n_tokens, head_dim / 2, base, row_pos);
   KV_COUNT_LAUNCH();
   KV_CUDA(cudaGetLastError());
   return KV_OK;

@@ -200,11 +200,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
         // chunks c and c + d/64.  The row is token `row` of the call, at absolute position pos0 + row.
         const int d = qa.head_dim, half = d >> 1, pair = d >> 6;
         const bool live = row < m;
-        const int pos = qa.pos0 + row;
         long long slot_off = 0;
         int block = 0;
         if (live) {
-          block = qa.block_table[pos / qa.cache.block_size];
+          const int pos = qa.row_pos != nullptr ? qa.row_pos[row] : qa.pos0 + row;
+          block = qa.row_block != nullptr ? qa.row_block[row] : qa.block_table[pos / qa.cache.block_size];
           slot_off = (long long)(pos % qa.cache.block_size) * qa.cache.n_kv_heads * d;
         }
         const float2 *cs_row = qa.rope + (long long)row * half;

@@ -139,6 +139,13 @@ def test_prefill_and_decode_rejections(kv):
     assert prefill(ws=_FakeBuf(need, 0x7300000010)) == O.ERR_WORKSPACE
     wide = synth.ModelShape(**{**s.__dict__, "n_kv_heads": 4})
     assert prefill(cache=_FakeCache(kv, wide, 12)) == O.ERR_SHAPE
+    # batched form: tables are checked per request and block ids across the whole batch
+    def batched(id_lists, tabs):
+        return _status(kv.kv_prefill_prefix_batched, M, cache, id_lists, tabs, workspace=ws, stream=0)
+    assert batched([ids[:20], ids[:30]], [[3, 1], [4]]) == O.ERR_TABLE_SHORT        # 30 tokens need 2 blocks
+    assert batched([ids[:20], ids[:30]], [[3, 1], [4, 3]]) == O.ERR_BLOCK_ALIAS     # block 3 used by both requests
+    assert batched([ids[:20], ids[:30]], [[3, 1], [4, 12]]) == O.ERR_BLOCK_RANGE
+    assert batched([ids[:20], [s.vocab] * 3], [[3, 1], [4]]) == O.ERR_TOKEN_RANGE
     dneed = kv.kv_workspace_bytes(M, kv.KV_OP_DECODE, 64)
     dws = _FakeBuf(dneed, 0x7300000000)
     logits = _FakeBuf(4 * s.vocab, 0x7400000000)

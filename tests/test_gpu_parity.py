@@ -359,3 +359,38 @@ def test_chunked_prefill_wide_shape_tensor_core_path(kv, torch):
     sl = error_stats(lg2.cpu().numpy(), lg1.cpu().numpy())
     print("chunked vs single-shot:", st, sl)
     assert st["rel_l2"] <= 5e-3 and sl["rel_l2"] <= 1e-2, (st, sl)
+
+
+@pytest.mark.parametrize("name,layers,lengths", [("tiny-sharp", 2, (100, 37, 260)), ("32b", 2, (512, 300))])
+def test_batched_prefill_equals_separate_calls(kv, torch, name, layers, lengths):
+    """Several prefix reconstructions in one call: every page and the per-request logits must be identical to
+    separate calls (rows of a projection do not depend on the other rows in the launch; attention runs per request)."""
+    s = synth.SHAPES[name].with_layers(layers)
+    s = synth.ModelShape(**{**s.__dict__, "vocab": min(s.vocab, 2048)})
+    head = synth.head_weights(s, 9)
+    model = kv.Model(s, head, lambda l: synth.layer_weights(s, 9, l))
+    perm = synth.block_permutation(10, 256)
+    ids, tables, used = [], [], 0
+    for i, n in enumerate(lengths):
+        ids.append(synth.token_ids(s, 20 + i, n))
+        nb = -(-n // s.block_size)
+        tables.append(perm[used:used + nb].copy())
+        used += nb
+    one = kv.PagedCache(s, 256, fill=0)
+    two = kv.PagedCache(s, 256, fill=0)
+    lg_sep = torch.zeros(len(lengths), s.vocab, dtype=torch.float32, device="cuda")
+    lg_bat = torch.zeros_like(lg_sep)
+    for i in range(len(lengths)):
+        ws = kv.kv_prefill_prefix(model, one, ids[i], tables[i], logits_out=lg_sep[i])
+        kv.kv_check_device_status(ws)
+    ws = kv.kv_prefill_prefix_batched(model, two, ids, tables, logits_out=lg_bat)
+    kv.kv_check_device_status(ws)
+    torch.cuda.synchronize()
+    assert torch.equal(one.data, two.data)
+    assert bool(one.data.any())
+    assert torch.equal(lg_sep, lg_bat)
+    # K/V-only form (last layer stops after its K/V): same pages
+    three = kv.PagedCache(s, 256, fill=0)
+    kv.kv_prefill_prefix_batched(model, three, ids, tables)
+    torch.cuda.synchronize()
+    assert torch.equal(one.data, three.data)
