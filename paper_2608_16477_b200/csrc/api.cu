@@ -17,6 +17,17 @@ void set_cuda_error(cudaError_t e, const char *what) {
 
 long long g_launches = 0;
 
+int sm_count(int device) {
+  static int cached[kMaxDevices] = {};
+  if (device < 0 || device >= kMaxDevices) return 148;
+  if (cached[device] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || n <= 0) n = 148;
+    cached[device] = n;
+  }
+  return cached[device];
+}
+
 // ---- optional event profiler: CUDA events around each kernel class, on the caller's stream ----
 struct ProfRecord {
   int kind;

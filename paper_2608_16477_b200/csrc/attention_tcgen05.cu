@@ -399,8 +399,11 @@ int attention_prefill_tc(const bf16 *qkv_ctx, int n_tokens, int pos0, int n_q_he
   CUtensorMap map;
   int rc = tc::make_tmap_2d(&map, qkv_ctx, pos0 + n_tokens, qkv_dim, qkv_dim, kBM);
   if (rc != KV_OK) return rc;
-  static int regs_ok = -1;
-  if (regs_ok < 0) {
+  static int regs_ok_dev[kMaxDevices] = {};   // 0: not checked, 1: ok, 2: unbalanced
+  const int device = current_device();
+  if (device < 0) return KV_ERR_CUDA;
+  if (regs_ok_dev[device] == 0) {
+    int regs_ok;
     KV_CUDA(cudaFuncSetAttribute(attention_prefill_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  AttnSmem<64>::kBytes));
     KV_CUDA(cudaFuncSetAttribute(attention_prefill_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -416,8 +419,9 @@ int attention_prefill_tc(const bf16 *qkv_ctx, int n_tokens, int pos0, int n_q_he
       const int softmax_threads = kAttnThreads - 128;
       if (compiled < kRegsOther || softmax_threads * (kRegsSoftmax - compiled) > 128 * (compiled - kRegsOther)) regs_ok = 0;
     }
+    regs_ok_dev[device] = regs_ok ? 1 : 2;
   }
-  if (regs_ok == 0) return KV_ERR_SHAPE;
+  if (regs_ok_dev[device] != 1) return KV_ERR_SHAPE;
   const int m_tiles = (n_tokens + kBM - 1) / kBM;
   const int grid = m_tiles * (n_q_heads / 2);
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)head_dim);

@@ -61,6 +61,16 @@ enum ProfKind {
     }                                                  \
   } while (0)
 
+// Per-device one-time set-up (opt-in shared-memory sizes, SM counts): function attributes belong to a device,
+// so the "done" state is kept per device ordinal, not per process.
+constexpr int kMaxDevices = 64;
+inline int current_device() {
+  int device = 0;
+  if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kMaxDevices) return -1;
+  return device;
+}
+int sm_count(int device);   // multiprocessors of `device` (cached)
+
 // ---- launchers implemented in the .cu files (all enqueue on `st` and return a status) ----
 enum GemmMode { GEMM_STORE_BF16 = 0, GEMM_RESID_F32 = 1, GEMM_SWIGLU = 2, GEMM_QKV_ROPE = 3 };
 

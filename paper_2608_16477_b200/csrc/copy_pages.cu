@@ -129,16 +129,17 @@ __global__ void __launch_bounds__(kCopyThreads) copy_pages_kernel(const __grid_c
 
 int copy_pages(CacheView cache, int n_layers, const int *ids_host, int n_blocks, char *wire, int wire_layout,
                int total_blocks_in_wire, int first_block_in_wire, bool to_wire, cudaStream_t st) {
-  static int sms = 0;
-  if (sms == 0) {
-    int device = 0;
-    KV_CUDA(cudaGetDevice(&device));
-    KV_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+  static bool attr_set[kMaxDevices] = {};
+  const int device = current_device();
+  if (device < 0) return KV_ERR_CUDA;
+  if (!attr_set[device]) {
     KV_CUDA(cudaFuncSetAttribute(copy_pages_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kBufs * kPieceBytes));
     KV_CUDA(cudaFuncSetAttribute(copy_pages_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kBufs * kPieceBytes));
+    attr_set[device] = true;
   }
+  const int sms = sm_count(device);
   for (int done = 0; done < n_blocks; done += kMaxIds) {
     PageCopyParams p;
     p.cache = cache;

@@ -59,7 +59,7 @@ __global__ void __launch_bounds__(kGemvWarps * 32) gemv2_kernel(const bf16 *__re
                                                                 int k, float *__restrict__ y,
                                                                 const __grid_constant__ GemvQkvArgs qa) {
   const int lane = threadIdx.x & 31;
-  const int unit = blockIdx.x * kGemvWarps + (threadIdx.x >> 5);
+  const int unit = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   int row_a, row_b;
   bool has_b = true;
   if (EPI == GEMV_SWIGLU) {
@@ -160,8 +160,12 @@ template <int EPI, bool NORM>
 static int launch_gemv2(const bf16 *w, const float *x, const bf16 *gain, float eps, int n, int k, float *y,
                         const GemvQkvArgs &qa, cudaStream_t st) {
   const int units = (EPI == GEMV_SWIGLU) ? n : (n + 1) / 2;
-  const int grid = (units + kGemvWarps - 1) / kGemvWarps;
-  gemv2_kernel<EPI, NORM><<<grid, kGemvWarps * 32, 0, st>>>(w, x, gain, eps, n, k, y, qa);
+  // warps per CTA: few enough that every SM gets at least ~8 CTAs, so the SMs finish together even when
+  // a product has only a few thousand row pairs (O, down and QKV projections)
+  int warps = units / (sm_count(current_device()) * 8);
+  warps = warps < 1 ? 1 : (warps > kGemvWarps ? kGemvWarps : warps);
+  const int grid = (units + warps - 1) / warps;
+  gemv2_kernel<EPI, NORM><<<grid, warps * 32, 0, st>>>(w, x, gain, eps, n, k, y, qa);
   KV_COUNT_LAUNCH();
   KV_CUDA(cudaGetLastError());
   return KV_OK;

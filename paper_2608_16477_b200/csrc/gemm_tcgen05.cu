@@ -350,11 +350,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
 template <int MODE, int BN>
 int launch_gemm(const CUtensorMap &ta, const CUtensorMap &tb, int m, int n, int k, bf16 *out, float *resid,
                 DeviceStatus *status, const QkvRopeArgs &qa, int sms, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
+  static bool attr_set[kMaxDevices] = {};
+  const int device = current_device();
+  if (device < 0) return KV_ERR_CUDA;
+  if (!attr_set[device]) {
     KV_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<MODE, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  TileCfg<MODE, BN>::kSmemBytes));
-    attr_set = true;
+    attr_set[device] = true;
   }
   const int out_cols = (MODE == GEMM_SWIGLU) ? BN / 2 : BN;
   const int tiles = ((m + BM - 1) / BM) * ((n + out_cols - 1) / out_cols);
@@ -405,12 +407,7 @@ int gemm_tc(const bf16 *a, int lda, const bf16 *w, int m, int n, int k, int mode
   }
   if ((k % 8) != 0 || (lda % 8) != 0 || (n % 8) != 0) return KV_ERR_SHAPE;
   if (((uintptr_t)a & 15) || ((uintptr_t)w & 15)) return KV_ERR_ARG;
-  static int sms = 0;
-  if (sms == 0) {
-    int device = 0;
-    KV_CUDA(cudaGetDevice(&device));
-    KV_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
-  }
+  const int sms = sm_count(current_device());
   const int bn = pick_bn(m, n, sms, mode, mode == GEMM_QKV_ROPE ? qa.head_dim : 0);
   CUtensorMap ta, tb;
   int rc = tc::make_tmap_2d(&ta, a, m, k, lda, BM);
