@@ -201,7 +201,9 @@ int32_t kv_unpack_blocks_batched(const kv_cache_desc *dst, int32_t n_req, const 
  * mode 0: out_dev bf16 [M, N] = A W^T.
  * mode 1: resid_dev fp32 [M, N] += A W^T (residual stream update).
  * mode 2: W is [2N, K] (gate | up); out_dev bf16 [M, N] = silu(A Wg^T) * (A Wu^T)  (SwiGLU).
- * K must be a multiple of 64 and N of 16.  M is arbitrary. */
+ * K and N must be multiples of 8.  M is arbitrary.  mode | KV_GEMM_CTA_PAIR selects the kernel in which two CTAs
+ * (two SMs) share one 256 x 256 tile through tcgen05 cta_group::2; results are identical. */
+#define KV_GEMM_CTA_PAIR 0x100
 int32_t kv_op_gemm(const void *a_dev, int32_t lda, const void *w_dev, int32_t m, int32_t n, int32_t k,
                    int32_t mode, void *out_dev, float *resid_dev, int32_t *status_dev, void *stream);
 

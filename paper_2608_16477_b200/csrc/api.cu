@@ -1,5 +1,6 @@
 // C ABI: argument validation on the host, workspace carving and the launch sequences of the four operations.
 #include <algorithm>
+#include <cstdlib>
 #include <cstring>
 #include <string>
 #include <vector>
@@ -236,8 +237,21 @@ long long wire_bytes_needed(const kv_cache_desc *c, int n_blocks) {
   return (long long)n_blocks * c->n_layers * 2 * c->block_size * c->n_kv_heads * c->head_dim * 2;
 }
 
+// Which projections run on the CTA-pair kernel (bit mask over GemmMode), settable for experiments through
+// the KV_GEMM_PAIR_MODES environment variable; rows below one pair tile always use the one-CTA kernel.
+int pair_mode_mask() {
+  static int mask = -1;
+  if (mask < 0) {
+    const char *e = getenv("KV_GEMM_PAIR_MODES");
+    mask = e ? atoi(e) : ((1 << GEMM_SWIGLU) | (1 << GEMM_QKV_ROPE));
+  }
+  return mask;
+}
+
 int run_gemm(const kv_model *, const bf16 *a, int lda, const bf16 *w, int rows, int n, int k, int mode, bf16 *out,
              float *resid, DeviceStatus *status, cudaStream_t st, const QkvRopeArgs *qa = nullptr) {
+  if (rows >= 256 && ((pair_mode_mask() >> mode) & 1))
+    return gemm_tc_pair(a, lda, w, rows, n, k, mode, out, resid, reinterpret_cast<int *>(status), st, qa);
   return gemm_tc(a, lda, w, rows, n, k, mode, out, resid, reinterpret_cast<int *>(status), st, qa);
 }
 
@@ -620,8 +634,13 @@ int32_t kv_unpack_blocks_batched(const kv_cache_desc *dst, int32_t n_req, const 
 
 int32_t kv_op_gemm(const void *a_dev, int32_t lda, const void *w_dev, int32_t m, int32_t n, int32_t k, int32_t mode,
                    void *out_dev, float *resid_dev, int32_t *status_dev, void *stream) {
+  const bool pair = (mode & KV_GEMM_CTA_PAIR) != 0;
+  mode &= ~KV_GEMM_CTA_PAIR;
   if (a_dev == nullptr || w_dev == nullptr || mode < 0 || mode > 2) return KV_ERR_ARG;
   if ((mode == GEMM_RESID_F32 && resid_dev == nullptr) || (mode != GEMM_RESID_F32 && out_dev == nullptr)) return KV_ERR_ARG;
+  if (pair)
+    return gemm_tc_pair((const bf16 *)a_dev, lda, (const bf16 *)w_dev, m, n, k, mode, (bf16 *)out_dev, resid_dev,
+                        status_dev, (cudaStream_t)stream);
   return gemm_tc((const bf16 *)a_dev, lda, (const bf16 *)w_dev, m, n, k, mode, (bf16 *)out_dev, resid_dev, status_dev,
                  (cudaStream_t)stream);
 }

@@ -86,6 +86,9 @@ struct QkvRopeArgs {
 
 int gemm_tc(const bf16 *a, int lda, const bf16 *w, int m, int n, int k, int mode, bf16 *out,
             float *resid, int *status_dev, cudaStream_t st, const QkvRopeArgs *qkv_args = nullptr);
+// CTA-pair (cta_group::2) variant with 256 x 256 tiles; same contract
+int gemm_tc_pair(const bf16 *a, int lda, const bf16 *w, int m, int n, int k, int mode, bf16 *out, float *resid,
+                 int *status_dev, cudaStream_t st, const QkvRopeArgs *qkv_args = nullptr);
 int gemm_simt(const bf16 *a, int lda, const bf16 *w, int m, int n, int k, int mode, bf16 *out,
               float *resid, cudaStream_t st);
 

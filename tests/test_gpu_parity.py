@@ -153,6 +153,28 @@ def test_gemm_tensor_core(kv, torch, m, n, k, mode):
         assert np.max(np.abs(got - want)) <= tol, error_stats(got, want)
 
 
+@pytest.mark.parametrize("m,n,k", [(256, 256, 64), (300, 520, 192), (1000, 1048, 512), (4096, 5120, 256)])
+@pytest.mark.parametrize("mode", [0, 1, 2])
+def test_gemm_cta_pair_identical_to_single_cta(kv, torch, m, n, k, mode):
+    """The cta_group::2 kernel (two SMs per 256-row tile) accumulates in the same order as the one-CTA kernel."""
+    g = torch.Generator(device="cuda").manual_seed(m + n + k + mode)
+    a = torch.empty(m, k, dtype=torch.bfloat16, device="cuda").normal_(0.0, 1.0, generator=g)
+    w = torch.empty(2 * n if mode == 2 else n, k, dtype=torch.bfloat16, device="cuda").normal_(0.0, 0.05, generator=g)
+    r0 = torch.randn(m, n, device="cuda", generator=g)
+    status = torch.zeros(64, dtype=torch.int32, device="cuda")
+    res = []
+    for flag in (0, 0x100):
+        out = torch.zeros(m, n, dtype=torch.bfloat16, device="cuda")
+        resid = r0.clone()
+        kv.kv_op_gemm(a, w, mode | flag, out=None if mode == 1 else out, resid=resid if mode == 1 else None,
+                      status=status, n=n)
+        torch.cuda.synchronize()
+        res.append(resid if mode == 1 else out)
+    assert int(status[0]) == 0, status[:8].tolist()
+    assert torch.equal(res[0], res[1])
+    assert bool(res[0].float().abs().sum() > 0)
+
+
 def test_gemm_matches_cuda_core_crosscheck(kv, torch):
     rng = np.random.default_rng(5)
     a = torch.from_numpy(rng.standard_normal((384, 320), dtype=np.float32)).cuda().to(torch.bfloat16)
