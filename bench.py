@@ -46,7 +46,7 @@ WORKLOADS = {
 
 # DRAM bytes (read + write) of one gate/up GEMM launch at the 32b-4k workload, from the ncu capture
 # summarised under profiles/ (same shape as the bench's launch: M 4096, K 5120, 2 x 25600 weight rows).
-NCU_TRAFFIC_BYTES = {"32b-4k": 857.2e6}   # profiles/gemm_tc_gate_up_32b-4k.md: 653.7 MB read + 203.5 MB written
+NCU_TRAFFIC_BYTES = {"32b-4k": 1264.3e6}   # profiles/gemm_tc_pair_gate_up_32b-4k.md: 1,057.2 MB read + 207.1 MB written
 
 
 def peaks():
@@ -353,7 +353,7 @@ def run_ours(args):
     gu_flops = 2.0 * prefix * shape.hidden * 2 * shape.ffn
     achieved = gu_flops / (gu_ms / max(gu_launches, 1) * 1e-3) / 1e12 if gu_ms > 0 else 0.0
     flops = prefill_flops(shape, prefix)
-    roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel<SWIGLU> (gate/up projection)", "achieved": achieved,
+    roofline = {"bound": "tensor", "kernel": "gemm_tc_pair_kernel<SWIGLU, 256> (gate/up projection, cta_group::2)", "achieved": achieved,
                 "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": achieved / pk["bf16_tflops_sustained"],
                 "frac_of_burst_peak": achieved / pk["bf16_tflops"], "peak_source": pk["source"] + " (sustained)",
                 "flops_per_launch": gu_flops, "launches_timed": gu_launches,

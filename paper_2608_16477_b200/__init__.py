@@ -11,6 +11,6 @@ from .binding import (KVError, load, lib_path, status_string, Model, PagedCache,
                       kv_window_waste_bound, kv_ewma, kv_op_gemm, kv_op_gemm_reference, kv_op_gemv, kv_op_rmsnorm,
                       kv_op_attention_prefill, kv_op_paged_attention, kv_op_paged_attention_noalloc, kv_paged_attention_scratch_bytes,
                       kv_fill_pattern, kv_profile_enable, kv_profile_read, kv_launch_count, PROFILE_KINDS, EXPORTS, KV_OP_PREFILL, KV_OP_DECODE, KV_WIRE_BLOCK_MAJOR,
-                      KV_WIRE_LAYER_MAJOR)
+                      KV_WIRE_LAYER_MAJOR, KV_GEMM_CTA_PAIR)
 
 __all__ = [n for n in dir() if not n.startswith("_")]

@@ -320,9 +320,18 @@ def kv_unpack_blocks_batched(cache, blk_offsets, dst_block_ids, wires, wire_layo
     _batched("kv_unpack_blocks_batched", cache, blk_offsets, dst_block_ids, wires, wire_layout, stream)
 
 
+KV_GEMM_CTA_PAIR = 0x100
+
+
 def kv_op_gemm(a, w, mode: int, out=None, resid=None, status=None, stream=None, n=None):
+    """mode 0 store / 1 residual add / 2 SwiGLU, optionally | KV_GEMM_CTA_PAIR for the two-SM kernel."""
     m, k = a.shape
-    n = n if n is not None else (w.shape[0] // 2 if mode == 2 else w.shape[0])
+    base_mode = mode & ~KV_GEMM_CTA_PAIR
+    n = n if n is not None else (w.shape[0] // 2 if base_mode == 2 else w.shape[0])
+    want = (m, n)
+    for t in (out, resid):
+        if t is not None and hasattr(t, "shape") and tuple(t.shape) != want:
+            raise ValueError(f"output shape {tuple(t.shape)} does not match the product's {want}")
     _check(load().kv_op_gemm(_ptr(a), a.stride(0), _ptr(w), m, n, k, mode, _ptr(out), _ptr(resid), _ptr(status),
                              _stream(stream)), "kv_op_gemm")
 

@@ -23,6 +23,7 @@ def main():
     ap.add_argument("--tokens", type=int, default=4096)
     ap.add_argument("--iters", type=int, default=3)
     ap.add_argument("--blocks", type=int, default=32, help="pack/unpack: blocks per launch")
+    ap.add_argument("--pair", action="store_true", help="GEMM cases: the CTA-pair (cta_group::2) kernel")
     a = ap.parse_args()
     kv.load()
     s = synth.SHAPES[a.shape]
@@ -51,7 +52,8 @@ def main():
             out, resid, flops = torch.empty(t, s.qkv_dim, dtype=torch.bfloat16, device=dev), None, 2.0 * t * s.hidden * s.qkv_dim
         else:
             raise SystemExit(f"unknown case {a.case}")
-        run = lambda: kv.kv_op_gemm(x, w, mode, out=out, resid=resid, status=status)
+        flag = 0x100 if a.pair else 0     # KV_GEMM_CTA_PAIR
+        run = lambda: kv.kv_op_gemm(x, w, mode | flag, out=out, resid=resid, status=status)
         work, unit = flops / 1e12, "TFLOP/s"
     elif a.case == "attention":
         qkv = rnd(t, s.qkv_dim)
