@@ -258,13 +258,13 @@ int launch_pair(const CUtensorMap &ta, const CUtensorMap &tb, int m, int n, int 
 
 // Tile width minimising waves x width / efficiency over the SM pairs (same model as the one-CTA kernel).
 int pick_bn_pair(int m, int n_out, int sms, int mode, int head_dim) {
-  const int widths[4] = {256, 224, 192, 160};
-  const double eff[4] = {1.00, 0.97, 0.92, 0.85};
+  const int widths[5] = {256, 224, 192, 160, 128};
+  const double eff[5] = {1.00, 0.97, 0.92, 0.88, 0.85};
   const long long m_tiles = (m + 2 * BM - 1) / (2 * BM);
   const int pairs = sms / 2;
   int best = 256;
   double best_cost = -1.0;
-  for (int i = 0; i < 4; ++i) {
+  for (int i = 0; i < 5; ++i) {
     const int bn = widths[i];
     if (mode == GEMM_QKV_ROPE && (bn % head_dim) != 0) continue;
     if (mode == GEMM_SWIGLU && (bn % 64) != 0) continue;
@@ -310,14 +310,18 @@ int gemm_tc_pair(const bf16 *a, int lda, const bf16 *w, int m, int n, int k, int
   KV_PAIR_CASE(GEMM_RESID_F32, 224);
   KV_PAIR_CASE(GEMM_RESID_F32, 192);
   KV_PAIR_CASE(GEMM_RESID_F32, 160);
+  KV_PAIR_CASE(GEMM_RESID_F32, 128);
   KV_PAIR_CASE(GEMM_STORE_BF16, 256);
   KV_PAIR_CASE(GEMM_STORE_BF16, 224);
   KV_PAIR_CASE(GEMM_STORE_BF16, 192);
   KV_PAIR_CASE(GEMM_STORE_BF16, 160);
+  KV_PAIR_CASE(GEMM_STORE_BF16, 128);
   KV_PAIR_CASE(GEMM_SWIGLU, 256);
   KV_PAIR_CASE(GEMM_SWIGLU, 192);
+  KV_PAIR_CASE(GEMM_SWIGLU, 128);
   KV_PAIR_CASE(GEMM_QKV_ROPE, 256);
   KV_PAIR_CASE(GEMM_QKV_ROPE, 192);
+  KV_PAIR_CASE(GEMM_QKV_ROPE, 128);
 #undef KV_PAIR_CASE
   return KV_ERR_ARG;
 }
