@@ -10,11 +10,14 @@ reconstructed and positions [k, n) are covered it assembles the merged block tab
 
 Every byte is moved by kv_pack_blocks / kv_unpack_assemble; this module only sequences streams, events and
 metadata.  `LoopbackTransport` delivers into a receiver on the same GPU (a device-to-device copy stands in for
-the link); a two-GPU transport would replace that copy by a send/receive of the same wire slot into the
-receiver's own memory.
+the link).  `PeerTransport` is the two-process form: the sender issues one point-to-point send of a small
+header and one of the wire slot per block (torch.distributed; NCCL over NVLink between two GPUs), and the
+receiver posts the matching receive straight into its own receive buffer, so the payload lands in the target's
+memory before any kernel of the target reads it.
 """
 from __future__ import annotations
 
+import contextlib
 from collections import deque
 from dataclasses import dataclass
 
@@ -47,18 +50,31 @@ class SuffixReceiver:
     def slot(self, i):
         return self.buffer[i * self.block_elems:(i + 1) * self.block_elems]
 
+    def accepts(self, request_id: int, epoch: int) -> bool:
+        """Whether an arriving block belongs to this migration attempt and still has a slot; a refused block
+        counts as dropped."""
+        ok = (epoch == self.expected_epoch and request_id == self.request_id
+              and (len(self.logical) + 1) * self.block_elems <= self.buffer.numel())
+        if not ok:
+            self.dropped += 1
+        return ok
+
+    def next_slot(self):
+        """The receive-buffer slot the next accepted block lands in."""
+        return self.slot(len(self.logical))
+
+    def commit(self, logical_block: int) -> None:
+        """Records that the slot returned by next_slot() now holds `logical_block`."""
+        self.logical.append(int(logical_block))
+
     def on_block(self, msg: BlockMessage, copy_stream) -> bool:
         """Stores one arriving block; returns False when it is discarded (stale epoch, foreign request, no room)."""
         import torch
-        if msg.epoch != self.expected_epoch or msg.request_id != self.request_id:
-            self.dropped += 1
-            return False
-        if len(self.logical) * self.block_elems >= self.buffer.numel():
-            self.dropped += 1
+        if not self.accepts(msg.request_id, msg.epoch):
             return False
         with torch.cuda.stream(copy_stream):
-            self.slot(len(self.logical)).copy_(msg.wire, non_blocking=True)     # stands in for the link
-        self.logical.append(int(msg.logical_block))
+            self.next_slot().copy_(msg.wire, non_blocking=True)     # stands in for the link
+        self.commit(msg.logical_block)
         return True
 
     def assemble(self, prefix_table, n_tokens_total: int, epoch: int, stream=None):
@@ -79,6 +95,68 @@ class LoopbackTransport:
     def send(self, msg: BlockMessage, stream) -> None:
         self.receiver.on_block(msg, stream)
         self.sent_blocks += 1
+
+
+def _on_stream(stream):
+    import torch
+    return torch.cuda.stream(stream) if stream is not None else contextlib.nullcontext()
+
+
+class PeerTransport:
+    """Point-to-point transport between the source's process and the target's (one process per GPU).
+
+    Sender: `send(msg, stream)` enqueues, in stream order after the pack that filled the wire slot, a 4-word
+    header (kind, request id, epoch, logical block) and the slot itself; `close(stream)` sends the end-of-stream
+    header.  Receiver: `recv_into(receiver, stream)` takes one header, then receives the payload directly into
+    the receiver's next buffer slot, or into a scratch slot when the receiver refuses the block (stale epoch,
+    foreign request, buffer full), so that sends and receives always pair up.  Tensors live wherever the
+    process group's backend expects them (device memory for NCCL, host memory for gloo); the transport moves
+    bytes and metadata only.
+    """
+
+    KIND_BLOCK, KIND_END = 0, 1
+
+    def __init__(self, peer: int, group=None):
+        self.peer, self.group = int(peer), group
+        self.sent_blocks = 0
+        self._scratch = None
+
+    def _header(self, like, kind, request_id=0, epoch=0, logical_block=0):
+        import torch
+        return torch.tensor([kind, request_id, epoch, logical_block], dtype=torch.int64, device=like.device)
+
+    def send(self, msg: BlockMessage, stream=None) -> None:
+        import torch.distributed as dist
+        with _on_stream(stream):
+            dist.send(self._header(msg.wire, self.KIND_BLOCK, msg.request_id, msg.epoch, msg.logical_block),
+                      self.peer, group=self.group)
+            dist.send(msg.wire, self.peer, group=self.group)
+        self.sent_blocks += 1
+
+    def close(self, like, stream=None) -> None:
+        """Tells the receiver that no further block follows (`like`: any tensor on the sending device)."""
+        import torch.distributed as dist
+        with _on_stream(stream):
+            dist.send(self._header(like, self.KIND_END), self.peer, group=self.group)
+
+    def recv_into(self, receiver: SuffixReceiver, stream=None):
+        """Receives one message.  Returns True (block stored), False (block dropped) or None (end of stream)."""
+        import torch
+        import torch.distributed as dist
+        with _on_stream(stream):
+            header = torch.empty(4, dtype=torch.int64, device=receiver.buffer.device)
+            dist.recv(header, self.peer, group=self.group)
+            kind, request_id, epoch, logical_block = (int(v) for v in header.tolist())   # waits for the header
+            if kind == self.KIND_END:
+                return None
+            if receiver.accepts(request_id, epoch):
+                dist.recv(receiver.next_slot(), self.peer, group=self.group)
+                receiver.commit(logical_block)
+                return True
+            if self._scratch is None:
+                self._scratch = torch.empty_like(receiver.slot(0))
+            dist.recv(self._scratch, self.peer, group=self.group)
+            return False
 
 
 class SuffixStreamer:
