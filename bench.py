@@ -95,11 +95,31 @@ def blas_threads():
         return os.cpu_count()
 
 
-def cpu_baseline(shape, prefix, sample_tokens, repeats=1):
+def oracle_copy_rates(shape, n_blocks):
+    """The oracle's pack and unpack/assemble over n_blocks scattered pages, in GB/s (bytes read + bytes written)."""
+    from oracle import kv_oracle as O
+    pool = 2 * n_blocks + 8
+    cache = O.new_cache(shape.n_layers, pool, shape.block_size, shape.n_kv_heads, shape.head_dim, fill=1)
+    ids = np.random.default_rng(5).permutation(pool)
+    src, dst = ids[:n_blocks], ids[n_blocks:2 * n_blocks]
+    t0 = time.perf_counter()
+    wire = O.pack_blocks(cache, src)
+    t1 = time.perf_counter()
+    st, _ = O.unpack_assemble(cache, wire, np.arange(n_blocks), dst, [], n_blocks * shape.block_size)
+    t2 = time.perf_counter()
+    assert st == O.OK
+    return 2.0 * wire.nbytes / (t1 - t0) / 1e9, 2.0 * wire.nbytes / (t2 - t1) / 1e9
+
+
+def cpu_baseline(shape, prefix, sample_tokens, repeats=1, suffix_blocks=0):
     run = oracle_sample(shape, sample_tokens)
     secs = min(run() for _ in range(repeats))
     value = sample_tokens / (secs * shape.n_layers)
-    return {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+    extra = {}
+    if suffix_blocks:
+        pack, unpack = oracle_copy_rates(shape, suffix_blocks)
+        extra = {"pack_gbs": pack, "unpack_gbs": unpack, "copy_sample": f"{suffix_blocks} suffix blocks, one thread"}
+    return {**extra, "value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
             "sample": f"one decoder layer (1 of {shape.n_layers}) of the fp64 numpy oracle over the first "
                       f"{sample_tokens} of {prefix} prefix tokens, {secs:.2f} s; tokens/s extrapolated to "
                       f"{shape.n_layers} layers",
@@ -387,7 +407,8 @@ def run_ours(args):
         "breakdown_ms_per_step": {k: round(v[0], 4) for k, v in per_step.items()},
     }
     if world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = cpu_baseline(synth.SHAPES[shape_name], prefix, min(prefix, args.ref_tokens))
+        line["cpu_baseline"] = cpu_baseline(synth.SHAPES[shape_name], prefix, min(prefix, args.ref_tokens),
+                                            suffix_blocks=-(-suffix // synth.SHAPES[shape_name].block_size))
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
