@@ -3,19 +3,22 @@
 // prefix (gathered from its pages), rows [pos0, pos0 + T) the chunk's post-RoPE Q, K and V.
 //
 // One CTA works on ONE 128-row query tile of TWO query heads that share a KV head (tiles "a" and "b"), so
-// every K/V tile fetched by TMA feeds both, and the two softmax warpgroups alternate with the tensor core:
-// while one tile's scores are being exponentiated, the other tile's MMAs run.
+// every K/V tile fetched by TMA feeds both.
 //
-//   warp 0      TMA producer: Q tiles once, then K and V tiles (128 keys) into a 2-stage ring.
+//   warp 0      TMA producer of Q (once) and of the K tiles (128 keys each); warp 2: producer of the V tiles.
 //   warp 1      TMEM allocation and MMA issue:  S = Q K^T  (both operands K-major in shared memory),
 //               O += P V  (P read from TMEM, V as an MN-major shared-memory operand: no transposes).
 //   warps 4-7   softmax of tile a, warps 8-11 softmax of tile b: one thread per query row (= TMEM lane).
 //               The row of S is read once into registers (setmaxnreg moves registers from warps 0-3 to the
-//               softmax warps), reduced to its maximum and turned into bf16 probabilities written back over
-//               the first half of S in TMEM.  Statistics stay in fp32; the running maximum is
-//               only advanced (and O rescaled in TMEM) when it grows by more than 8 in the log2 domain,
-//               which keeps exp2 arguments <= 8 and makes rescaling rare.
-// TMEM columns: S_a [0,128)  S_b [128,256)  O_a [256,256+D)  O_b [384,384+D).
+//               softmax warps) and the S columns are handed back at once: the two tiles take turns on ONE
+//               score buffer, and each has its own columns for the bf16 probabilities, so the scores of a
+//               tile's NEXT key tile are computed while this one is exponentiated.
+//               Statistics stay in fp32; the running maximum is only advanced (and O rescaled in TMEM) when
+//               it grows by more than 8 in the log2 domain, which keeps exp2 arguments <= 8 and makes
+//               rescaling rare.
+// Per key tile a softmax warpgroup therefore waits only for things issued most of a step earlier (S of this
+// tile, P V of the previous one); the tensor pipe and the exponentials overlap instead of alternating.
+// TMEM columns: S [0,128)  P_a [128,192)  P_b [192,256)  O_a [256,256+D)  O_b [384,384+D).
 // Tiles are launched heaviest-first (causal work grows with the row tile index).
 // Every mbarrier wait is bounded; a wait that runs out is recorded in the status block and the CTA drains.
 #include "tc_common.cuh"
@@ -26,9 +29,8 @@ namespace {
 
 constexpr int kBM = 128;            // query rows per tile
 constexpr int kBN = 128;            // keys per KV tile
-constexpr int kKvStages = 2;
 constexpr int kAttnThreads = 384;   // 12 warps
-constexpr uint32_t kTmemS0 = 0, kTmemS1 = 128, kTmemO0 = 256, kTmemO1 = 384;
+constexpr uint32_t kTmemS = 0, kTmemP0 = 128, kTmemP1 = 192, kTmemO0 = 256, kTmemO1 = 384;
 constexpr float kRescaleThreshold = 8.0f;
 // setmaxnreg moves registers inside the pool the CTA was launched with (threads x registers per thread as
 // compiled), and setmaxnreg.inc blocks, with no timeout, until the registers it asks for have been released.
@@ -45,16 +47,9 @@ __device__ long long g_attn_trace[64 * 16];
 #define KV_ATRACE(slot, idx) do { } while (0)
 #endif
 
-enum AttnTag { ATAG_Q = 11, ATAG_KV_EMPTY = 12, ATAG_K = 13, ATAG_V = 14, ATAG_S = 15, ATAG_P = 16, ATAG_O = 17 };
+enum AttnTag { ATAG_Q = 11, ATAG_K_EMPTY = 12, ATAG_K = 13, ATAG_V = 14, ATAG_S = 15, ATAG_P = 16, ATAG_O = 17,
+               ATAG_V_EMPTY = 18, ATAG_S_FREE = 19, ATAG_PV = 20 };
 
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-      : "memory");
-}
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
@@ -64,6 +59,15 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
         "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
         "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
 }
 
@@ -84,12 +88,16 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   return *reinterpret_cast<uint32_t *>(&h);
 }
 
+// Shared memory: two Q tiles, a ring of K tiles and a ring of V tiles.
 template <int D>
 struct AttnSmem {
+  static constexpr int kKStages = 2;
+  static constexpr int kVStages = 2;
   static constexpr int kTileBytes = kBM * D * 2;                 // one Q, K or V tile
-  static constexpr int kQOff = 0;                                // 2 Q tiles
-  static constexpr int kKvOff = 2 * kTileBytes;                  // stages of (K, V)
-  static constexpr int kBarOff = kKvOff + kKvStages * 2 * kTileBytes;
+  static constexpr int kQOff = 0;
+  static constexpr int kKOff = 2 * kTileBytes;
+  static constexpr int kVOff = kKOff + kKStages * kTileBytes;
+  static constexpr int kBarOff = kVOff + kVStages * kTileBytes;
   static constexpr int kBytes = kBarOff + 256 + 1024;            // barriers + alignment slack
 };
 
@@ -100,14 +108,15 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
   using L = AttnSmem<D>;
   constexpr int kAtoms = D / 64;                   // 64-column (128-byte) boxes per tile row
   constexpr int kBoxBytes = kBM * 128;             // one 128-row x 64-col box
+  constexpr int kKS = L::kKStages, kVS = L::kVStages;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t *smem_gen = smem_raw + (smem_base - tc::smem_u32(smem_raw));
   const uint32_t bar_base = smem_base + L::kBarOff;
-  // barriers: q_full[2] k_full[2] v_full[2] kv_empty[2] s_full[2] p_ready[2] o_full[2]
+  // barriers, two of each: Q full, K full, V full, K empty, V empty, S full, S free, P ready, P V done
+  enum { B_Q = 0, B_K = 1, B_V = 2, B_K_EMPTY = 3, B_V_EMPTY = 4, B_S = 5, B_S_FREE = 6, B_P = 7, B_PV = 8, B_GROUPS = 9 };
   auto bar = [&](int group, int idx) { return bar_base + 8u * (group * 2 + idx); };
-  enum { B_Q = 0, B_K = 1, B_V = 2, B_KV_EMPTY = 3, B_S = 4, B_P = 5, B_O = 6 };
-  uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(smem_gen + L::kBarOff + 8 * 14);
+  uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(smem_gen + L::kBarOff + 8 * 2 * B_GROUPS);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -131,10 +140,12 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
       tc::mbar_init(bar(B_Q, i), 1);
       tc::mbar_init(bar(B_K, i), 1);
       tc::mbar_init(bar(B_V, i), 1);
-      tc::mbar_init(bar(B_KV_EMPTY, i), 1);
+      tc::mbar_init(bar(B_K_EMPTY, i), 1);
+      tc::mbar_init(bar(B_V_EMPTY, i), 1);
       tc::mbar_init(bar(B_S, i), 1);
+      tc::mbar_init(bar(B_S_FREE, i), 128);
       tc::mbar_init(bar(B_P, i), 128);
-      tc::mbar_init(bar(B_O, i), 1);
+      tc::mbar_init(bar(B_PV, i), 1);
     }
     *abort_flag = 0;
     tc::fence_barrier_init();
@@ -148,7 +159,7 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
   // the softmax warpgroups hold a full row of S in registers; warps 0-3 give registers back (first statement
   // of every role so the register budget of each branch is known at compile time)
   if (warp == 0) {
-    // ---------------------------------------------------------------- TMA producer
+    // ---------------------------------------------------------------- TMA producer: Q, then the K tiles
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
     if (lane == 0) {
       tc::tma_prefetch_desc(&tma_qkv);
@@ -159,70 +170,98 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
                           bar(B_Q, t));
       }
       for (int j = 0; j < n_kv; ++j) {
-        const int st = j & 1;
-        const uint32_t ph = (j >> 1) & 1;
-        if (!tc::mbar_wait(bar(B_KV_EMPTY, st), ph ^ 1, abort_flag, status, ATAG_KV_EMPTY)) break;
-        const uint32_t k_s = smem_base + L::kKvOff + st * 2 * L::kTileBytes;
-        const uint32_t v_s = k_s + L::kTileBytes;
+        const int st = j % kKS;
+        const uint32_t ph = (j / kKS) & 1;
+        if (!tc::mbar_wait(bar(B_K_EMPTY, st), ph ^ 1, abort_flag, status, ATAG_K_EMPTY)) break;
+        const uint32_t k_s = smem_base + L::kKOff + st * L::kTileBytes;
         tc::mbar_expect_tx(bar(B_K, st), L::kTileBytes);
         for (int a = 0; a < kAtoms; ++a)
           tc::tma_load_2d(k_s + a * kBoxBytes, &tma_qkv, k_col + a * 64, j * kBN, bar(B_K, st));
+      }
+    }
+  } else if (warp == 2) {
+    // ---------------------------------------------------------------- TMA producer: the V tiles
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
+    if (lane == 0) {
+      for (int j = 0; j < n_kv; ++j) {
+        const int st = j % kVS;
+        const uint32_t ph = (j / kVS) & 1;
+        if (!tc::mbar_wait(bar(B_V_EMPTY, st), ph ^ 1, abort_flag, status, ATAG_V_EMPTY)) break;
+        const uint32_t v_s = smem_base + L::kVOff + st * L::kTileBytes;
         tc::mbar_expect_tx(bar(B_V, st), L::kTileBytes);
         for (int a = 0; a < kAtoms; ++a)
           tc::tma_load_2d(v_s + a * kBoxBytes, &tma_qkv, v_col + a * 64, j * kBN, bar(B_V, st));
       }
     }
   } else if (warp == 1) {
-    // ---------------------------------------------------------------- MMA issuer
+    // ---------------------------------------------------------------- MMA issuer: S = Q K^T
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
-    if (lane == 0) {
+    {
+      // every lane waits, and the verdict is made uniform so that the warp stays converged for elect.sync
+      auto wwait = [&](uint32_t b_, uint32_t parity, volatile int *af, DeviceStatus *st_, int tag) {
+        return __all_sync(0xffffffffu, tc::mbar_wait(b_, parity, af, st_, tag)) != 0;
+      };
       constexpr uint32_t idesc_qk = tc::umma_idesc_bf16(kBM, kBN);
-      constexpr uint32_t idesc_pv = tc::umma_idesc_bf16(kBM, D) | (1u << 16);   // B (= V) is MN-major
-      const uint32_t s_tmem[2] = {tmem_base + kTmemS0, tmem_base + kTmemS1};
-      const uint32_t o_tmem[2] = {tmem_base + kTmemO0, tmem_base + kTmemO1};
+      const uint32_t s_tmem = tmem_base + kTmemS;
       auto issue_qk = [&](int t, int st) {
         const uint32_t q_s = smem_base + L::kQOff + t * L::kTileBytes;
-        const uint32_t k_s = smem_base + L::kKvOff + st * 2 * L::kTileBytes;
+        const uint32_t k_s = smem_base + L::kKOff + st * L::kTileBytes;
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
           const uint32_t off = (ks / 4) * kBoxBytes + (ks % 4) * 32;
-          tc::umma_bf16(s_tmem[t], tc::umma_desc_k128(q_s + off), tc::umma_desc_k128(k_s + off), idesc_qk, ks != 0);
+          tc::umma_bf16_warp(s_tmem, tc::umma_desc_k128(q_s + off), tc::umma_desc_k128(k_s + off), idesc_qk, ks != 0);
         }
-        tc::umma_commit(bar(B_S, t));
+        tc::umma_commit_warp(bar(B_S, t));
       };
-      bool ok = tc::mbar_wait(bar(B_Q, 0), 0, abort_flag, status, ATAG_Q) &&
-                tc::mbar_wait(bar(B_Q, 1), 0, abort_flag, status, ATAG_Q) &&
-                tc::mbar_wait(bar(B_K, 0), 0, abort_flag, status, ATAG_K);
-      if (ok) {
-        tc::tc_fence_after();
-        issue_qk(0, 0);
-        issue_qk(1, 0);
-      }
+      // The score buffer is used in the order a_0 b_0 a_1 b_1 ...: each use starts once the previous user
+      // has taken its scores into registers (S free).
+      bool ok = wwait(bar(B_Q, 0), 0, abort_flag, status, ATAG_Q) &&
+                wwait(bar(B_Q, 1), 0, abort_flag, status, ATAG_Q);
       for (int j = 0; j < n_kv && ok; ++j) {
-        const int st = j & 1;
-        const uint32_t ph = (j >> 1) & 1;
-        const uint32_t v_s = smem_base + L::kKvOff + st * 2 * L::kTileBytes + L::kTileBytes;
+        const int kst = j % kKS;
+        ok = wwait(bar(B_K, kst), (j / kKS) & 1, abort_flag, status, ATAG_K);
         for (int t = 0; t < 2 && ok; ++t) {
-          ok = tc::mbar_wait(bar(B_P, t), j & 1, abort_flag, status, ATAG_P) &&
-               tc::mbar_wait(bar(B_V, st), ph, abort_flag, status, ATAG_V);
+          // before use 2j + t of the buffer, use 2j + t - 1 must have been read: that is tile 1 - t
+          if (j + t > 0) ok = wwait(bar(B_S_FREE, t ^ 1), (t == 0 ? j - 1 : j) & 1, abort_flag, status, ATAG_S_FREE);
           if (!ok) break;
-          KV_ATRACE(8 + t * 2, j);
+          tc::tc_fence_after();
+          if (t == 0 && lane == 0) KV_ATRACE(9, j);
+          issue_qk(t, kst);
+          if (t == 0 && lane == 0) KV_ATRACE(11, j);
+        }
+        if (!ok) break;
+        tc::umma_commit_warp(bar(B_K_EMPTY, kst));
+      }
+    }
+  } else if (warp == 3) {
+    // ---------------------------------------------------------------- MMA issuer: O += P V
+    // (its own thread: issuing one tcgen05.mma costs this thread more cycles than a 128 x 128 x 16 MMA runs)
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
+    {
+      auto wwait = [&](uint32_t b_, uint32_t parity, volatile int *af, DeviceStatus *st_, int tag) {
+        return __all_sync(0xffffffffu, tc::mbar_wait(b_, parity, af, st_, tag)) != 0;
+      };
+      constexpr uint32_t idesc_pv = tc::umma_idesc_bf16(kBM, D) | (1u << 16);   // B (= V) is MN-major
+      const uint32_t p_tmem[2] = {tmem_base + kTmemP0, tmem_base + kTmemP1};
+      const uint32_t o_tmem[2] = {tmem_base + kTmemO0, tmem_base + kTmemO1};
+      bool ok = true;
+      for (int j = 0; j < n_kv && ok; ++j) {
+        const int vst = j % kVS;
+        ok = wwait(bar(B_V, vst), (j / kVS) & 1, abort_flag, status, ATAG_V);
+        const uint32_t v_s = smem_base + L::kVOff + vst * L::kTileBytes;
+        for (int t = 0; t < 2 && ok; ++t) {
+          ok = wwait(bar(B_P, t), j & 1, abort_flag, status, ATAG_P);
+          if (!ok) break;
+          if (lane == 0) KV_ATRACE(8 + 2 * t, j);
           tc::tc_fence_after();
 #pragma unroll
           for (int ks = 0; ks < kBN / 16; ++ks)   // 16 keys per slice: 8 TMEM columns of P, 2048 bytes of V
-            tc::umma_bf16_ts(o_tmem[t], s_tmem[t] + ks * 8, umma_desc_mn128(v_s + ks * 2048, kBoxBytes), idesc_pv,
+            tc::umma_bf16_ts_warp(o_tmem[t], p_tmem[t] + ks * 8, umma_desc_mn128(v_s + ks * 2048, kBoxBytes), idesc_pv,
                              (j | ks) != 0);
-          if (t == 1) tc::umma_commit(bar(B_KV_EMPTY, st));
-          if (j + 1 < n_kv) {
-            ok = tc::mbar_wait(bar(B_K, st ^ 1), ((j + 1) >> 1) & 1, abort_flag, status, ATAG_K);
-            if (!ok) break;
-            tc::tc_fence_after();
-            issue_qk(t, st ^ 1);
-          } else {
-            tc::umma_commit(bar(B_O, t));
-          }
-          KV_ATRACE(9 + t * 2, j);
+          tc::umma_commit_warp(bar(B_PV, t));
         }
+        if (!ok) break;
+        tc::umma_commit_warp(bar(B_V_EMPTY, vst));
       }
     }
   } else if (warp < 4) {
@@ -235,7 +274,8 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
     const int row_in_tile = quarter * 32 + lane;
     const int qi = pos0 + m0 + row_in_tile;        // absolute query position
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-    const uint32_t s_t = tmem_base + lane_base + (t == 0 ? kTmemS0 : kTmemS1);
+    const uint32_t s_t = tmem_base + lane_base + kTmemS;
+    const uint32_t p_t = tmem_base + lane_base + (t == 0 ? kTmemP0 : kTmemP1);
     const uint32_t o_t = tmem_base + lane_base + (t == 0 ? kTmemO0 : kTmemO1);
     float m_ref = -INFINITY, l_sum = 0.f;
     bool ok = true;
@@ -247,13 +287,15 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
       tc::tc_fence_after();
       const bool diag = (j * kBN + kBN - 1 > pos0 + m0);   // tile reaches past the first row's position
       const int limit = qi - j * kBN;              // keys with column > limit are masked
-      // the whole row of S (128 fp32) in registers: four loads in flight, one wait
+      // the whole row of S (128 fp32) in registers: four loads in flight, one wait; then S may be overwritten
       uint32_t r0[32], r1[32], r2[32], r3[32];
       tc::tmem_ld32(s_t + 0, r0);
       tc::tmem_ld32(s_t + 32, r1);
       tc::tmem_ld32(s_t + 64, r2);
       tc::tmem_ld32(s_t + 96, r3);
       tc::tmem_ld_wait();
+      tc::tc_fence_before();
+      tc::mbar_arrive(bar(B_S_FREE, t));
       if (quarter == 0 && lane == 0) KV_ATRACE(t * 4 + 1, j);
       float mx = -INFINITY;
       if (!diag) {
@@ -284,8 +326,34 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
         m_ref = mx;
         l_sum *= factor;
       }
+      if (quarter == 0 && lane == 0) KV_ATRACE(t * 4 + 2, j);
+      // probabilities as packed bf16 (two keys per 32-bit column); masked scores are -inf -> 0.  The first half
+      // of the row is exponentiated before the wait for the P columns, so that the wait finds P V_{j-1} done.
+      const float neg_m = -m_ref;
+      float sum0 = 0.f, sum1 = 0.f;
+      auto exps = [&](const uint32_t (&r)[32], uint32_t (&pk)[16]) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const float p0 = exp2f(fmaf(__uint_as_float(r[2 * i]), scale_log2, neg_m));
+          const float p1 = exp2f(fmaf(__uint_as_float(r[2 * i + 1]), scale_log2, neg_m));
+          sum0 += p0;
+          sum1 += p1;
+          pk[i] = pack2(p0, p1);
+        }
+      };
+      auto store = [&](const uint32_t (&pk)[16], int c) { tmem_st16(p_t + c * 16, pk); };   // 32 keys
+      uint32_t pk0[16], pk1[16];
+      exps(r0, pk0);
+      exps(r1, pk1);
+      // P V of the previous key tile must be done before its P columns are overwritten or O is rescaled
+      if (j > 0) {
+        ok = tc::mbar_wait(bar(B_PV, t), (j - 1) & 1, abort_flag, status, ATAG_PV);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc::tc_fence_after();
+      }
+      if (quarter == 0 && lane == 0) KV_ATRACE(12 + t, j);
       if (__any_sync(0xffffffffu, rescale)) {
-        // O of this tile is idle: the MMAs that produced S_j were issued after PV_{j-1}
 #pragma unroll 1
         for (int c = 0; c < D / 32; ++c) {
           uint32_t r[32];
@@ -296,26 +364,15 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
           tmem_st32(o_t + c * 32, r);
         }
       }
-      if (quarter == 0 && lane == 0) KV_ATRACE(t * 4 + 2, j);
-      // probabilities, written over S as packed bf16 (two keys per 32-bit column); masked scores are -inf -> 0
-      const float neg_m = -m_ref;
-      float sum0 = 0.f, sum1 = 0.f;
-      auto emit = [&](const uint32_t (&r)[32], int c) {
+      store(pk0, 0);
+      store(pk1, 1);
+      {
         uint32_t pk[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const float p0 = exp2f(fmaf(__uint_as_float(r[2 * i]), scale_log2, neg_m));
-          const float p1 = exp2f(fmaf(__uint_as_float(r[2 * i + 1]), scale_log2, neg_m));
-          sum0 += p0;
-          sum1 += p1;
-          pk[i] = pack2(p0, p1);
-        }
-        tmem_st16(s_t + c * 16, pk);
-      };
-      emit(r0, 0);
-      emit(r1, 1);
-      emit(r2, 2);
-      emit(r3, 3);
+        exps(r2, pk);
+        store(pk, 2);
+        exps(r3, pk);
+        store(pk, 3);
+      }
       l_sum += sum0 + sum1;
       tc::tmem_st_wait();
       tc::tc_fence_before();
@@ -323,7 +380,7 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
       if (quarter == 0 && lane == 0) KV_ATRACE(t * 4 + 3, j);
     }
     if (ok) {
-      ok = tc::mbar_wait(bar(B_O, t), 0, abort_flag, status, ATAG_O);
+      ok = tc::mbar_wait(bar(B_PV, t), (n_kv - 1) & 1, abort_flag, status, ATAG_O);
       ok = __all_sync(0xffffffffu, ok);
     }
     if (ok) {

@@ -129,7 +129,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // The whole warp runs the loop and one elected lane issues each instruction: operands prepared per warp
+    // reach tcgen05.mma far faster than from a single-lane branch.
+    {
+      auto wwait = [&](uint32_t b_, uint32_t parity, int tag) {
+        return __all_sync(0xffffffffu, tc::mbar_wait(b_, parity, abort_flag, status, tag)) != 0;
+      };
       constexpr uint32_t idesc = tc::umma_idesc_bf16(BM, BN);
       int stage = 0;
       uint32_t phase = 0;
@@ -138,14 +143,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local) {
         const int buf = local & 1;
         const uint32_t acc_phase = (local >> 1) & 1;
-        KV_TRACE(1, local);
-        ok = tc::mbar_wait(tempty_bar(buf), acc_phase ^ 1, abort_flag, status, TAG_TMEM_EMPTY);
+        if (lane == 0) KV_TRACE(1, local);
+        ok = wwait(tempty_bar(buf), acc_phase ^ 1, TAG_TMEM_EMPTY);
         if (!ok) break;
-        KV_TRACE(2, local);
+        if (lane == 0) KV_TRACE(2, local);
         tc::tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * kTmemBufStride;
         for (int kb = 0; kb < k_blocks; ++kb) {
-          ok = tc::mbar_wait(full_bar(stage), phase, abort_flag, status, TAG_FULL);
+          ok = wwait(full_bar(stage), phase, TAG_FULL);
           if (!ok) break;
           tc::tc_fence_after();
           const uint32_t a_s = smem_base + stage * kStageBytes;
@@ -153,12 +158,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
           const uint64_t b_desc = tc::umma_desc_k128(a_s + kABytes);
 #pragma unroll
           for (int ks = 0; ks < BK / 16; ++ks)   // +32 bytes (2 descriptor units) per K=16 slice
-            tc::umma_bf16(d_tmem, a_desc + 2 * ks, b_desc + 2 * ks, idesc, (kb | ks) != 0);
-          tc::umma_commit(empty_bar(stage));
+            tc::umma_bf16_warp(d_tmem, a_desc + 2 * ks, b_desc + 2 * ks, idesc, (kb | ks) != 0);
+          tc::umma_commit_warp(empty_bar(stage));
           if (++stage == kStages) { stage = 0; phase ^= 1; }
         }
-        if (ok) tc::umma_commit(tfull_bar(buf));
-        KV_TRACE(3, local);
+        if (ok) tc::umma_commit_warp(tfull_bar(buf));
+        if (lane == 0) KV_TRACE(3, local);
       }
     }
   } else {
@@ -220,8 +225,14 @@ int launch_gemm(const CUtensorMap &ta, const CUtensorMap &tb, int m, int n, int 
 // M x N problem on `sms` SMs.  SwiGLU tiles hold a gate half and an up half, so a BN-wide tile yields BN / 2
 // output columns; QKV tiles must hold whole heads.
 int pick_bn(int m, int n_out, int sms, int mode, int head_dim) {
+  if (const char *e = getenv("KV_GEMM_BN")) {     // experiments: force one tile width where the mode allows it
+    const int bn = atoi(e);
+    const bool shape_ok = bn >= 128 && bn <= 256 && bn % 32 == 0 &&
+                          !(mode == GEMM_QKV_ROPE && (bn % head_dim) != 0) && !(mode == GEMM_SWIGLU && (bn % 64) != 0);
+    if (shape_ok) return bn;
+  }
   const int widths[5] = {256, 224, 192, 160, 128};
-  const double eff[5] = {1.00, 0.97, 0.92, 0.85, 0.75};     // measured: narrower tiles re-read A more often and
+  const double eff[5] = {1.00, 1.00, 0.99, 0.96, 0.85};     // measured: narrower tiles re-read A more often and
                                                              // amortise the per-stage barrier work over fewer flops
   const long long m_tiles = (m + BM - 1) / BM;
   int best = 256;

@@ -78,18 +78,23 @@ __device__ __forceinline__ void tmem_alloc_pair(uint32_t holder_smem, uint32_t n
 __device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
   asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
+// Whole-warp forms (every lane calls with the same operands, one elected lane issues).
 __device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                                uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
+      "{\n\t.reg .pred pe, p;\n\t"
+      "elect.sync _|pe, 0xffffffff;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      "@pe tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 // one arrival on the mbarrier at `bar_cluster` (own or peer CTA) once all MMAs issued so far are done
 __device__ __forceinline__ void umma_commit_pair(uint32_t bar_cluster) {
-  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_cluster) : "memory");
+  asm volatile(
+      "{\n\t.reg .pred pe;\n\t"
+      "elect.sync _|pe, 0xffffffff;\n\t"
+      "@pe tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(bar_cluster) : "memory");
 }
 
 template <int MODE, int BN>
@@ -167,7 +172,10 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_cons
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA only)
-    if (lane == 0 && rank == 0) {
+    if (rank == 0) {
+      auto wwait = [&](uint32_t b_, uint32_t parity, int tag) {
+        return __all_sync(0xffffffffu, tc::mbar_wait(b_, parity, abort_flag, status, tag)) != 0;
+      };
       constexpr uint32_t idesc = tc::umma_idesc_bf16(2 * BM, BN);
       int stage = 0;
       uint32_t phase = 0;
@@ -176,12 +184,12 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_cons
       for (int tile = pair; tile < total_tiles && ok; tile += n_pairs, ++local) {
         const int buf = local & 1;
         const uint32_t acc_phase = (local >> 1) & 1;
-        ok = tc::mbar_wait(tempty_bar(buf), acc_phase ^ 1, abort_flag, status, TAG2_TMEM_EMPTY);
+        ok = wwait(tempty_bar(buf), acc_phase ^ 1, TAG2_TMEM_EMPTY);
         if (!ok) break;
         tc::tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * kTmemBufStride;
         for (int kb = 0; kb < k_blocks; ++kb) {
-          ok = tc::mbar_wait(full_bar(stage), phase, abort_flag, status, TAG2_FULL);
+          ok = wwait(full_bar(stage), phase, TAG2_FULL);
           if (!ok) break;
           tc::tc_fence_after();
           const uint32_t a_s = smem_base + stage * kStageBytes;
@@ -258,8 +266,14 @@ int launch_pair(const CUtensorMap &ta, const CUtensorMap &tb, int m, int n, int 
 
 // Tile width minimising waves x width / efficiency over the SM pairs (same model as the one-CTA kernel).
 int pick_bn_pair(int m, int n_out, int sms, int mode, int head_dim) {
+  if (const char *e = getenv("KV_GEMM_BN")) {     // experiments: force one tile width where the mode allows it
+    const int bn = atoi(e);
+    const bool shape_ok = bn >= 128 && bn <= 256 && bn % 32 == 0 &&
+                          !(mode == GEMM_QKV_ROPE && (bn % head_dim) != 0) && !(mode == GEMM_SWIGLU && (bn % 64) != 0);
+    if (shape_ok) return bn;
+  }
   const int widths[5] = {256, 224, 192, 160, 128};
-  const double eff[5] = {1.00, 0.97, 0.92, 0.88, 0.85};
+  const double eff[5] = {1.00, 0.99, 0.98, 0.92, 0.78};     // measured per-column cost relative to 256-wide tiles
   const long long m_tiles = (m + 2 * BM - 1) / (2 * BM);
   const int pairs = sms / 2;
   int best = 256;
