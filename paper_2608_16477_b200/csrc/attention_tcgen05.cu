@@ -5,9 +5,11 @@
 // One CTA works on ONE 128-row query tile of TWO query heads that share a KV head (tiles "a" and "b"), so
 // every K/V tile fetched by TMA feeds both.
 //
-//   warp 0      TMA producer of Q (once) and of the K tiles (128 keys each); warp 2: producer of the V tiles.
-//   warp 1      TMEM allocation and MMA issue:  S = Q K^T  (both operands K-major in shared memory),
-//               O += P V  (P read from TMEM, V as an MN-major shared-memory operand: no transposes).
+//   warp 0      TMA producer of Q (once) and of the K and V tiles (128 keys each).
+//   warps 1, 2  S = Q K^T of tile a and of tile b (both operands K-major in shared memory); warp 1 also
+//               allocates TMEM.  The whole warp runs the loop, one elected lane issues each tcgen05.mma.
+//   warp 3      O += P V of both tiles (P read from TMEM, V as an MN-major shared-memory operand: no
+//               transposes).
 //   warps 4-7   softmax of tile a, warps 8-11 softmax of tile b: one thread per query row (= TMEM lane).
 //               The row of S is read once into registers (setmaxnreg moves registers from warps 0-3 to the
 //               softmax warps) and the S columns are handed back at once: the two tiles take turns on ONE
@@ -40,9 +42,9 @@ constexpr int kRegsOther = 72;      // registers per thread of warps 0-3 after t
 constexpr int kRegsSoftmax = 216;   // registers per thread of the softmax warps
 
 #ifdef KV_ATTN_TRACE
-__device__ long long g_attn_trace[64 * 16];
+__device__ long long g_attn_trace[64 * 32];
 #define KV_ATRACE(slot, idx) \
-  do { if (blockIdx.x == 0 && (idx) < 64) g_attn_trace[(idx) * 16 + (slot)] = clock64(); } while (0)
+  do { if (blockIdx.x == 0 && (idx) < 64) g_attn_trace[(idx) * 32 + (slot)] = clock64(); } while (0)
 #else
 #define KV_ATRACE(slot, idx) do { } while (0)
 #endif
@@ -140,7 +142,7 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
       tc::mbar_init(bar(B_Q, i), 1);
       tc::mbar_init(bar(B_K, i), 1);
       tc::mbar_init(bar(B_V, i), 1);
-      tc::mbar_init(bar(B_K_EMPTY, i), 1);
+      tc::mbar_init(bar(B_K_EMPTY, i), 2);     // one arrival per Q K^T issuer
       tc::mbar_init(bar(B_V_EMPTY, i), 1);
       tc::mbar_init(bar(B_S, i), 1);
       tc::mbar_init(bar(B_S_FREE, i), 128);
@@ -159,7 +161,7 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
   // the softmax warpgroups hold a full row of S in registers; warps 0-3 give registers back (first statement
   // of every role so the register budget of each branch is known at compile time)
   if (warp == 0) {
-    // ---------------------------------------------------------------- TMA producer: Q, then the K tiles
+    // ---------------------------------------------------------------- TMA producer: Q, then K and V tiles
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
     if (lane == 0) {
       tc::tma_prefetch_desc(&tma_qkv);
@@ -169,32 +171,36 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
           tc::tma_load_2d(smem_base + L::kQOff + t * L::kTileBytes + a * kBoxBytes, &tma_qkv, q_col[t] + a * 64, pos0 + m0,
                           bar(B_Q, t));
       }
-      for (int j = 0; j < n_kv; ++j) {
+      auto load_k = [&](int j) {
         const int st = j % kKS;
-        const uint32_t ph = (j / kKS) & 1;
-        if (!tc::mbar_wait(bar(B_K_EMPTY, st), ph ^ 1, abort_flag, status, ATAG_K_EMPTY)) break;
+        if (!tc::mbar_wait(bar(B_K_EMPTY, st), ((j / kKS) & 1) ^ 1, abort_flag, status, ATAG_K_EMPTY)) return false;
         const uint32_t k_s = smem_base + L::kKOff + st * L::kTileBytes;
         tc::mbar_expect_tx(bar(B_K, st), L::kTileBytes);
         for (int a = 0; a < kAtoms; ++a)
           tc::tma_load_2d(k_s + a * kBoxBytes, &tma_qkv, k_col + a * 64, j * kBN, bar(B_K, st));
-      }
-    }
-  } else if (warp == 2) {
-    // ---------------------------------------------------------------- TMA producer: the V tiles
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
-    if (lane == 0) {
-      for (int j = 0; j < n_kv; ++j) {
+        return true;
+      };
+      auto load_v = [&](int j) {
         const int st = j % kVS;
-        const uint32_t ph = (j / kVS) & 1;
-        if (!tc::mbar_wait(bar(B_V_EMPTY, st), ph ^ 1, abort_flag, status, ATAG_V_EMPTY)) break;
+        if (!tc::mbar_wait(bar(B_V_EMPTY, st), ((j / kVS) & 1) ^ 1, abort_flag, status, ATAG_V_EMPTY)) return false;
         const uint32_t v_s = smem_base + L::kVOff + st * L::kTileBytes;
         tc::mbar_expect_tx(bar(B_V, st), L::kTileBytes);
         for (int a = 0; a < kAtoms; ++a)
           tc::tma_load_2d(v_s + a * kBoxBytes, &tma_qkv, v_col + a * 64, j * kBN, bar(B_V, st));
+        return true;
+      };
+      // in the order the tiles are consumed: K_0, then K_{j+1} before V_j
+      bool ok = load_k(0);
+      for (int j = 0; j < n_kv && ok; ++j) {
+        if (j + 1 < n_kv) ok = load_k(j + 1);
+        if (ok) ok = load_v(j);
       }
     }
-  } else if (warp == 1) {
-    // ---------------------------------------------------------------- MMA issuer: S = Q K^T
+  } else if (warp == 1 || warp == 2) {
+    // ---------------------------------------------------------------- MMA issuers: S = Q K^T, warp 1 for tile a,
+    // warp 2 for tile b.  While a warp issues tcgen05.mma with shared-memory operands, the other warps of its
+    // scheduler get fewer issue slots; one issuer per tile spreads that over two schedulers, and the P V issuer
+    // sits on a third.
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
     {
       // every lane waits, and the verdict is made uniform so that the warp stays converged for elect.sync
@@ -203,39 +209,31 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
       };
       constexpr uint32_t idesc_qk = tc::umma_idesc_bf16(kBM, kBN);
       const uint32_t s_tmem = tmem_base + kTmemS;
-      auto issue_qk = [&](int t, int st) {
-        const uint32_t q_s = smem_base + L::kQOff + t * L::kTileBytes;
-        const uint32_t k_s = smem_base + L::kKOff + st * L::kTileBytes;
+      const int t = warp - 1;
+      const uint32_t q_s = smem_base + L::kQOff + t * L::kTileBytes;
+      // The score buffer is used in the order a_0 b_0 a_1 b_1 ...: each use starts once the previous user
+      // (the other tile) has taken its scores into registers (S free).
+      bool ok = wwait(bar(B_Q, t), 0, abort_flag, status, ATAG_Q);
+      for (int j = 0; j < n_kv && ok; ++j) {
+        const int kst = j % kKS;
+        ok = wwait(bar(B_K, kst), (j / kKS) & 1, abort_flag, status, ATAG_K);
+        if (ok && j + t > 0) ok = wwait(bar(B_S_FREE, t ^ 1), (t == 0 ? j - 1 : j) & 1, abort_flag, status, ATAG_S_FREE);
+        if (!ok) break;
+        tc::tc_fence_after();
+        if (t == 0 && lane == 0) KV_ATRACE(9, j);
+        const uint32_t k_s = smem_base + L::kKOff + kst * L::kTileBytes;
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
           const uint32_t off = (ks / 4) * kBoxBytes + (ks % 4) * 32;
           tc::umma_bf16_warp(s_tmem, tc::umma_desc_k128(q_s + off), tc::umma_desc_k128(k_s + off), idesc_qk, ks != 0);
         }
         tc::umma_commit_warp(bar(B_S, t));
-      };
-      // The score buffer is used in the order a_0 b_0 a_1 b_1 ...: each use starts once the previous user
-      // has taken its scores into registers (S free).
-      bool ok = wwait(bar(B_Q, 0), 0, abort_flag, status, ATAG_Q) &&
-                wwait(bar(B_Q, 1), 0, abort_flag, status, ATAG_Q);
-      for (int j = 0; j < n_kv && ok; ++j) {
-        const int kst = j % kKS;
-        ok = wwait(bar(B_K, kst), (j / kKS) & 1, abort_flag, status, ATAG_K);
-        for (int t = 0; t < 2 && ok; ++t) {
-          // before use 2j + t of the buffer, use 2j + t - 1 must have been read: that is tile 1 - t
-          if (j + t > 0) ok = wwait(bar(B_S_FREE, t ^ 1), (t == 0 ? j - 1 : j) & 1, abort_flag, status, ATAG_S_FREE);
-          if (!ok) break;
-          tc::tc_fence_after();
-          if (t == 0 && lane == 0) KV_ATRACE(9, j);
-          issue_qk(t, kst);
-          if (t == 0 && lane == 0) KV_ATRACE(11, j);
-        }
-        if (!ok) break;
-        tc::umma_commit_warp(bar(B_K_EMPTY, kst));
+        tc::umma_commit_warp(bar(B_K_EMPTY, kst));      // second of the two arrivals frees the K stage
+        if (t == 0 && lane == 0) KV_ATRACE(11, j);
       }
     }
   } else if (warp == 3) {
     // ---------------------------------------------------------------- MMA issuer: O += P V
-    // (its own thread: issuing one tcgen05.mma costs this thread more cycles than a 128 x 128 x 16 MMA runs)
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
     {
       auto wwait = [&](uint32_t b_, uint32_t parity, volatile int *af, DeviceStatus *st_, int tag) {
@@ -249,6 +247,7 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
         const int vst = j % kVS;
         ok = wwait(bar(B_V, vst), (j / kVS) & 1, abort_flag, status, ATAG_V);
         const uint32_t v_s = smem_base + L::kVOff + vst * L::kTileBytes;
+        if (lane == 0) KV_ATRACE(24, j);
         for (int t = 0; t < 2 && ok; ++t) {
           ok = wwait(bar(B_P, t), j & 1, abort_flag, status, ATAG_P);
           if (!ok) break;
@@ -259,13 +258,12 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
             tc::umma_bf16_ts_warp(o_tmem[t], p_tmem[t] + ks * 8, umma_desc_mn128(v_s + ks * 2048, kBoxBytes), idesc_pv,
                              (j | ks) != 0);
           tc::umma_commit_warp(bar(B_PV, t));
+          if (lane == 0) KV_ATRACE(25 + t, j);
         }
         if (!ok) break;
         tc::umma_commit_warp(bar(B_V_EMPTY, vst));
       }
     }
-  } else if (warp < 4) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
   } else {
     // ---------------------------------------------------------------- softmax warpgroups
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
@@ -378,6 +376,7 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
       tc::tc_fence_before();
       tc::mbar_arrive(bar(B_P, t));
       if (quarter == 0 && lane == 0) KV_ATRACE(t * 4 + 3, j);
+      if (lane == 0) KV_ATRACE(16 + t * 4 + quarter, j);
     }
     if (ok) {
       ok = tc::mbar_wait(bar(B_PV, t), (n_kv - 1) & 1, abort_flag, status, ATAG_O);
@@ -496,7 +495,7 @@ int attention_prefill_tc(const bf16 *qkv_ctx, int n_tokens, int pos0, int n_q_he
 
 #ifdef KV_ATTN_TRACE
 extern "C" int kv_debug_attn_trace(long long *out_host) {
-  return cudaMemcpyFromSymbol(out_host, g_attn_trace, sizeof(long long) * 64 * 16) == cudaSuccess ? 0 : -13;
+  return cudaMemcpyFromSymbol(out_host, g_attn_trace, sizeof(long long) * 64 * 32) == cudaSuccess ? 0 : -13;
 }
 #endif
 
