@@ -46,7 +46,7 @@ WORKLOADS = {
 
 # DRAM bytes (read + write) of one gate/up GEMM launch at the 32b-4k workload, from the ncu capture
 # summarised under profiles/ (same shape as the bench's launch: M 4096, K 5120, 2 x 25600 weight rows).
-NCU_TRAFFIC_BYTES = {"32b-4k": 1264.3e6}   # profiles/gemm_tc_pair_gate_up_32b-4k.md: 1,057.2 MB read + 207.1 MB written
+NCU_TRAFFIC_BYTES = {"32b-4k": 1269.9e6}   # profiles/gemm_tc_pair_gate_up_32b-4k.md: 1,064.3 MB read + 205.6 MB written
 
 
 def peaks():
