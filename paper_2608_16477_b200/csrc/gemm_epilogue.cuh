@@ -113,18 +113,36 @@ __device__ __forceinline__ void gemm_epilogue_slab(uint32_t t_row, int row, int 
     // memory and a thread-per-row update would touch half a 32-byte sector per row and instruction.
     // Each warp therefore transposes 32 rows x 8 columns at a time through a 1 KiB shared-memory buffer
     // and updates x with two lanes per row: every instruction then moves whole 32-byte sectors of 16 rows.
+    // The old values of x for a 32-column slab (eight float4 per thread) are fetched one slab ahead, so the
+    // global-memory latency is paid once per tile instead of once per pass.
     float4 *stage = stage_base + (warp - 2) * 64;
     const int sub_row = lane >> 1, c4 = lane & 1;
+    auto x_ptr = [&](int c, int s8, int it) {
+      const int grow = m0 + quarter * 32 + it * 16 + sub_row;
+      const int scol = n0 + c * 32 + s8 * 8 + c4 * 4;
+      return (grow < m && scol < n) ? reinterpret_cast<float4 *>(resid + (long long)grow * n + scol) : nullptr;
+    };
+    auto fetch = [&](int c, float4 (&x)[8]) {
+#pragma unroll
+      for (int s8 = 0; s8 < 4; ++s8)
+#pragma unroll
+        for (int it = 0; it < 2; ++it) {
+          const float4 *px = x_ptr(c, s8, it);
+          x[s8 * 2 + it] = px != nullptr ? __ldcs(px) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    };
+    float4 x_cur[8], x_next[8];
+    fetch(0, x_cur);
 #pragma unroll 1
     for (int c = 0; c < BN / 32; ++c) {
       const int col = n0 + c * 32;
       if (col >= n) break;
+      if (c + 1 < BN / 32) fetch(c + 1, x_next);
       uint32_t r[32];
       tc::tmem_ld32(t_row + c * 32, r);
       tc::tmem_ld_wait();
 #pragma unroll
       for (int s8 = 0; s8 < 4; ++s8) {         // 8 columns per pass
-        const int scol = col + s8 * 8 + c4 * 4;
         // stage[row][2 chunks], chunk index XORed with bit 2 of the row: conflict-free both ways
         stage[lane * 2 + (0 ^ ((lane >> 2) & 1))] =
             make_float4(__uint_as_float(r[8 * s8]), __uint_as_float(r[8 * s8 + 1]), __uint_as_float(r[8 * s8 + 2]),
@@ -136,17 +154,18 @@ __device__ __forceinline__ void gemm_epilogue_slab(uint32_t t_row, int row, int 
 #pragma unroll
         for (int it = 0; it < 2; ++it) {
           const int rr = it * 16 + sub_row;
-          const int grow = m0 + quarter * 32 + rr;
-          if (grow < m && scol < n) {
+          float4 *px = x_ptr(c, s8, it);
+          if (px != nullptr) {
             const float4 a4 = stage[rr * 2 + (c4 ^ ((rr >> 2) & 1))];
-            float4 *px = reinterpret_cast<float4 *>(resid + (long long)grow * n + scol);
-            float4 x = __ldcs(px);
+            float4 x = x_cur[s8 * 2 + it];
             x.x += a4.x; x.y += a4.y; x.z += a4.z; x.w += a4.w;
             *px = x;
           }
         }
         __syncwarp();
       }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) x_cur[i] = x_next[i];
     }
   } else {
 #pragma unroll 1
