@@ -333,6 +333,16 @@ def run_ours(args):
     pack_ms, pack_how = graph_time(pack_all)
     unpack_ms, _ = graph_time(unpack_all)
 
+    # the decode step timed alone as well (direct launches), before the prefill pulls the clocks down
+    merged0 = kv.kv_unpack_assemble(tgt, wire, logical, dst_ids, tgt_prefix, n, epoch=1, expected_epoch=1)
+    table0 = list(merged0) + extra
+
+    def decode_only():
+        kv.kv_decode_step(model, tgt, int(ids[n]), n, table0, logits, workspace=ws_d)
+    for _ in range(3):
+        decode_only()
+    decode_alone_ms = timed(decode_only, 10) / 10
+
     for _ in range(max(args.warmup, 3)):
         step()
     kv.kv_check_device_status(ws_p)
@@ -403,6 +413,7 @@ def run_ours(args):
         "unpack": {"gbs": 2 * payload / (unpack_ms * 1e-3) / 1e9,
                    "frac_of_hbm": 2 * payload / (unpack_ms * 1e-3) / 1e9 / pk["hbm_gbs"], "us": unpack_ms * 1e3},
         "decode_step_ms": decode_ms,
+        "decode_step_alone_ms": decode_alone_ms,
         "t0_analog_ms": per_step["unpack"][0] + decode_ms,
         "breakdown_ms_per_step": {k: round(v[0], 4) for k, v in per_step.items()},
     }
