@@ -1,7 +1,7 @@
 """Runs ONE kernel of the hot path a few times at the benchmark's shapes, for profiler captures.
 
   python -m paper_2608_16477_b200.profile_case gemm_gate_up [--tokens 4096] [--iters 3]
-  cases: gemm_qkv, gemm_o, gemm_gate_up, gemm_down, attention, pack, unpack, decode_gemv
+  cases: gemm_qkv, gemm_o, gemm_gate_up, gemm_down, attention, pack, unpack, decode_gemv, decode_attention
 
 Inputs are synthetic and larger than L2 where the kernel is bandwidth-bound; a few GB at most are held on
 the device so a multi-pass capture stays short.  Prints the CUDA-event time per launch.
@@ -91,6 +91,27 @@ def main():
             state["i"] += 1
             kv.kv_op_gemv(ws[state["i"] % 4], x, 2, y, gain=gain, eps=1e-6)
         work, unit = ws[0].numel() * 2 / 1e9, "GB/s"
+    elif a.case == "decode_attention":
+        # one layer's paged attention of a decode step at context a.tokens + 512 (the bench's resume position),
+        # rotating over 4 layers of a fragmented cache so consecutive launches read cold pages
+        n_ctx = t + 512 + 1
+        pool = 1024
+        layers = 4
+        s4 = s.with_layers(layers)
+        cache = kv.PagedCache(s4, pool)
+        kv.kv_fill_pattern(cache.data, cache.data.numel() * 2, seed=1)
+        cache.data.bitwise_and_(0x3FFF)               # small finite bf16 values
+        table = torch.from_numpy(np.ascontiguousarray(synth.block_permutation(2, pool)[: -(-n_ctx // s.block_size)]
+                                                      .astype(np.int32))).to(dev)
+        q = torch.randn(s.n_q_heads, s.head_dim, device=dev)
+        out = torch.empty(s.n_q_heads, s.head_dim, device=dev)
+        scratch = torch.empty(kv.kv_paged_attention_scratch_bytes(s.n_q_heads, s.head_dim, n_ctx), dtype=torch.uint8, device=dev)
+        state = {"i": 0}
+
+        def run():
+            state["i"] += 1
+            kv.kv_op_paged_attention(q, cache, state["i"] % layers, table, n_ctx, scratch, out)
+        work, unit = 2.0 * n_ctx * s.n_kv_heads * s.head_dim * 2 / 1e9, "GB/s"
     else:
         raise SystemExit(f"unknown case {a.case}")
     run()
