@@ -208,15 +208,21 @@ int gemv_qkv_rope(const bf16 *w_qkv, const float *x, const bf16 *gain, float eps
 
 // ---- paged decode attention ---------------------------------------------------------------
 // Partial record per (q head, split): m, l, acc[d].
-// One CTA of 256 threads per (KV head, 256-key split), serving every query head of the group so each K/V
-// row is read from HBM once:
-//   phase 1  thread t loads the whole K row of key t (16-byte loads, all in flight at once) and scores it
-//            against the group's queries held in shared memory;
-//   phase 2  one warp per head: maximum, exponentials and their sum over the split's scores;
-//   phase 3  warp w walks keys 32w..32w+31, each lane owning d/32 dims of V, accumulating p * v for all
-//            heads; the eight warps' partial sums meet in shared memory.
-constexpr int kPaSplitKeys = 256;   // keys per split = threads per CTA
-constexpr int kPaHeadChunk = 8;     // query heads handled per pass over the keys
+// One CTA of 128 threads per (KV head, 128-key split), serving every query head of the group so each K/V
+// row is read from HBM once.  Thread t copies the K row and the V row of key t into shared memory with
+// 16-byte cp.async (everything in flight at once; 16-byte chunks XOR-swizzled by the row so that ldmatrix is
+// conflict-free).  The contractions run on mma.sync m16n8k16 (a 16-row tile is the natural size for the 8 to
+// 16 query heads of a group; the 128-row tcgen05 tile would be nine tenths padding):
+//   S = Q K^T   warp w owns keys 32w..32w+31; Q (fp32) is split into a bf16 high and low part, so the scores
+//               keep fp32-level accuracy at the cost of a second MMA;
+//   softmax     row maxima meet in shared memory, every warp then uses the split's common maximum;
+//   O = P V     P goes from the S accumulators straight into A fragments (again as high + low parts), V through
+//               ldmatrix.trans; the four warps' partial O and row sums are added in shared memory.
+constexpr int kPaSplitKeys = 128;   // keys per split = threads per CTA (two CTAs fit an SM)
+constexpr int kPaRows = 16;         // query heads per pass (rows of the MMA tile)
+
+// dynamic shared memory: the K and V tiles (2 x 128 rows of bf16) and 4 warps x 16 rows of fp32 partial O
+static int pa_smem_bytes(int d) { return 2 * kPaSplitKeys * d * 2 + (kPaSplitKeys / 32) * kPaRows * d * 4; }
 
 static int pa_splits(int n_ctx) {
   int s = (n_ctx + kPaSplitKeys - 1) / kPaSplitKeys;
@@ -227,40 +233,44 @@ long long paged_attention_scratch_bytes(int n_q_heads, int head_dim, int n_ctx) 
   return (long long)n_q_heads * pa_splits(n_ctx) * (head_dim + 2) * (long long)sizeof(float);
 }
 
-// DPL consecutive bf16 -> fp32 with one vector load (the address is DPL*2-byte aligned)
-template <int DPL>
-__device__ __forceinline__ void load_bf16(const bf16 *p, float (&out)[DPL]) {
-  static_assert(DPL == 2 || DPL == 4 || DPL == 8, "dims per lane");
-  if constexpr (DPL == 8) {
-    const uint4 raw = *reinterpret_cast<const uint4 *>(p);
-    const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&raw);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const float2 f = __bfloat1622float2(h[i]);
-      out[2 * i] = f.x;
-      out[2 * i + 1] = f.y;
-    }
-  } else if constexpr (DPL == 4) {
-    const uint2 raw = *reinterpret_cast<const uint2 *>(p);
-    const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&raw);
-    const float2 a = __bfloat1622float2(h[0]), b = __bfloat1622float2(h[1]);
-    out[0] = a.x; out[1] = a.y; out[2] = b.x; out[3] = b.y;
-  } else {
-    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(p));
-    out[0] = a.x; out[1] = a.y;
-  }
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+      "{%0, %1, %2, %3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+// x = hi + lo with hi = bf16(x), lo = bf16(x - hi): two bf16 that together carry ~16 mantissa bits
+__device__ __forceinline__ void split_pair(float x, float y, uint32_t &hi, uint32_t &lo) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(x, y);
+  const float2 hf = __bfloat1622float2(h);
+  const __nv_bfloat162 l = __floats2bfloat162_rn(x - hf.x, y - hf.y);
+  hi = *reinterpret_cast<const uint32_t *>(&h);
+  lo = *reinterpret_cast<const uint32_t *>(&l);
 }
 
 template <int D>
-__global__ void __launch_bounds__(kPaSplitKeys) paged_attention_split_kernel(
+__global__ void __launch_bounds__(kPaSplitKeys, 2) paged_attention_split_kernel(
     const float *__restrict__ q, int n_q_heads, CacheView cache, int layer, const int *__restrict__ block_table,
     int n_ctx, float *__restrict__ partial) {
-  constexpr int DPL = D / 32;
-  constexpr int HC = kPaHeadChunk;
-  __shared__ __align__(16) float q_s[HC][D];
-  __shared__ float p_s[HC][kPaSplitKeys];
-  __shared__ __align__(16) float red_s[kPaSplitKeys / 32][HC][D];
-  __shared__ float ml_s[HC][2];
+  constexpr int RB = D * 2;                 // bytes per K or V row
+  constexpr int CH = D / 8;                 // 16-byte chunks per row
+  constexpr int KS = D / 16;                // k-steps of S = Q K^T
+  constexpr int NT = D / 8;                 // n-tiles of O = P V
+  constexpr int NW = kPaSplitKeys / 32;     // warps
+  extern __shared__ __align__(128) uint8_t pa_smem[];
+  uint8_t *k_tile = pa_smem;                                  // [keys][D] bf16, swizzled
+  uint8_t *v_tile = pa_smem + kPaSplitKeys * RB;
+  float *o_red = reinterpret_cast<float *>(pa_smem + 2 * kPaSplitKeys * RB);   // [NW][kPaRows][D] partial O
+  __shared__ float wmax_s[NW][kPaRows], wsum_s[NW][kPaRows];
   const int g = blockIdx.x, split = blockIdx.y, n_splits = gridDim.y;
   const int group = n_q_heads / cache.n_kv_heads;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -268,124 +278,163 @@ __global__ void __launch_bounds__(kPaSplitKeys) paged_attention_split_kernel(
   const int j0 = split * kPaSplitKeys;
   const int n_keys = min(n_ctx - j0, kPaSplitKeys);
 
-  // this thread's key: K row into registers (phase 1 operand), V row address for later
-  const int jk = j0 + min(tid, n_keys - 1);
-  const long long row_off = ((long long)(jk % cache.block_size) * cache.n_kv_heads + g) * D;
-  const int blk_k = block_table[jk / cache.block_size];
-  uint4 kraw[D / 8];
+  // this thread's key (rows past the end repeat the last key: finite data, masked below)
   {
-    const uint4 *kp = reinterpret_cast<const uint4 *>(reinterpret_cast<const bf16 *>(cache.page(layer, 0, blk_k)) + row_off);
+    const int jk = j0 + min(tid, n_keys - 1);
+    const long long row_off = ((long long)(jk % cache.block_size) * cache.n_kv_heads + g) * D;
+    const int blk = block_table[jk / cache.block_size];
+    const bf16 *kp = reinterpret_cast<const bf16 *>(cache.page(layer, 0, blk)) + row_off;
+    const bf16 *vp = reinterpret_cast<const bf16 *>(cache.page(layer, 1, blk)) + row_off;
+    const uint32_t kd = (uint32_t)__cvta_generic_to_shared(k_tile + tid * RB);
+    const uint32_t vd = (uint32_t)__cvta_generic_to_shared(v_tile + tid * RB);
 #pragma unroll
-    for (int v = 0; v < D / 8; ++v) kraw[v] = kp[v];
+    for (int c = 0; c < CH; ++c) {
+      const uint32_t pc = (uint32_t)((c & ~7) | ((c ^ tid) & 7)) * 16;
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(kd + pc), "l"(kp + c * 8) : "memory");
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+#pragma unroll
+    for (int c = 0; c < CH; ++c) {
+      const uint32_t pc = (uint32_t)((c & ~7) | ((c ^ tid) & 7)) * 16;
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(vd + pc), "l"(vp + c * 8) : "memory");
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
   }
+  const uint32_t k_s = (uint32_t)__cvta_generic_to_shared(k_tile);
+  const uint32_t v_s = (uint32_t)__cvta_generic_to_shared(v_tile);
+  const int r0 = lane >> 2, cq = (lane & 3) * 2;       // fragment row (and row + 8), first of two columns
+  const int wk0 = warp * 32;                           // this warp's keys inside the split
 
-  for (int h0 = 0; h0 < group; h0 += HC) {
-    const int nh = min(HC, group - h0);
-    __syncthreads();   // previous chunk fully consumed
-    for (int e = tid; e < nh * D; e += kPaSplitKeys)
-      q_s[e / D][e % D] = q[(long long)(g * group + h0 + e / D) * D + e % D] * scale;
-    __syncthreads();
-    // ---- phase 1: scores of this thread's key against nh heads
+  for (int h0 = 0; h0 < group; h0 += kPaRows) {
+    const int nh = min(kPaRows, group - h0);
+    // Q fragments of rows r0 and r0 + 8 (heads h0 + row), scaled, as high and low bf16 parts
+    uint32_t qh[KS][4], ql[KS][4];
     {
-      float sc[HC];
+      const float *qa = q + (long long)(g * group + h0 + min(r0, nh - 1)) * D;
+      const float *qb = q + (long long)(g * group + h0 + min(r0 + 8, nh - 1)) * D;
+      const float sa = (r0 < nh) ? scale : 0.f, sb = (r0 + 8 < nh) ? scale : 0.f;
 #pragma unroll
-      for (int h = 0; h < HC; ++h) sc[h] = 0.f;
-#pragma unroll
-      for (int v = 0; v < D / 8; ++v) {
-        const __nv_bfloat162 *hk = reinterpret_cast<const __nv_bfloat162 *>(&kraw[v]);
-        const float2 k0 = __bfloat1622float2(hk[0]), k1 = __bfloat1622float2(hk[1]);
-        const float2 k2 = __bfloat1622float2(hk[2]), k3 = __bfloat1622float2(hk[3]);
-#pragma unroll
-        for (int h = 0; h < HC; ++h) {
-          if (h < nh) {
-            const float4 qa = *reinterpret_cast<const float4 *>(&q_s[h][v * 8]);
-            const float4 qb = *reinterpret_cast<const float4 *>(&q_s[h][v * 8 + 4]);
-            sc[h] += k0.x * qa.x + k0.y * qa.y + k1.x * qa.z + k1.y * qa.w + k2.x * qb.x + k2.y * qb.y + k3.x * qb.z +
-                     k3.y * qb.w;
-          }
-        }
-      }
-#pragma unroll
-      for (int h = 0; h < HC; ++h)
-        if (h < nh) p_s[h][tid] = (tid < n_keys) ? sc[h] : -FLT_MAX;
-    }
-    __syncthreads();
-    // ---- phase 2: warp h turns the scores of head h into exponentials
-    if (warp < nh) {
-      float v[kPaSplitKeys / 32];
-      float mx = -FLT_MAX;
-#pragma unroll
-      for (int i = 0; i < kPaSplitKeys / 32; ++i) {
-        v[i] = p_s[warp][lane + 32 * i];
-        mx = fmaxf(mx, v[i]);
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-      float sum = 0.f;
-#pragma unroll
-      for (int i = 0; i < kPaSplitKeys / 32; ++i) {
-        const float e = (lane + 32 * i < n_keys) ? __expf(v[i] - mx) : 0.f;
-        p_s[warp][lane + 32 * i] = e;
-        sum += e;
-      }
-      sum = warp_sum_d(sum);
-      if (lane == 0) {
-        ml_s[warp][0] = mx;
-        ml_s[warp][1] = sum;
+      for (int ks = 0; ks < KS; ++ks) {
+        const float2 a0 = *reinterpret_cast<const float2 *>(qa + ks * 16 + cq);
+        const float2 a2 = *reinterpret_cast<const float2 *>(qa + ks * 16 + 8 + cq);
+        const float2 b0 = *reinterpret_cast<const float2 *>(qb + ks * 16 + cq);
+        const float2 b2 = *reinterpret_cast<const float2 *>(qb + ks * 16 + 8 + cq);
+        split_pair(a0.x * sa, a0.y * sa, qh[ks][0], ql[ks][0]);
+        split_pair(b0.x * sb, b0.y * sb, qh[ks][1], ql[ks][1]);
+        split_pair(a2.x * sa, a2.y * sa, qh[ks][2], ql[ks][2]);
+        split_pair(b2.x * sb, b2.y * sb, qh[ks][3], ql[ks][3]);
       }
     }
-    __syncthreads();
-    // ---- phase 3: p * V, warp w over keys 32w .. 32w+31, lane owns DPL dims
-    {
-      float acc[HC][DPL];
+    if (h0 == 0) asm volatile("cp.async.wait_group 1;" ::: "memory");      // K rows have landed
+    __syncthreads();      // (also: the previous pass no longer reads o_red and the row statistics)
+    // ---- S = Q K^T for this warp's 32 keys: 4 n-tiles of 8 keys
+    float sc[4][4];
 #pragma unroll
-      for (int h = 0; h < HC; ++h)
+    for (int nt = 0; nt < 4; ++nt) {
 #pragma unroll
-        for (int i = 0; i < DPL; ++i) acc[h][i] = 0.f;
-      const int kb = warp * 32;
-      constexpr int U = 8;
-      for (int kk = 0; kk < 32 && kb + kk < n_keys; kk += U) {
-        float vf[U][DPL];
+      for (int i = 0; i < 4; ++i) sc[nt][i] = 0.f;
+      const int krow = wk0 + nt * 8 + (lane & 7);
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-          const int j = j0 + min(kb + kk + u, n_keys - 1);
-          const int blk = block_table[j / cache.block_size];
-          const bf16 *vp = reinterpret_cast<const bf16 *>(cache.page(layer, 1, blk)) +
-                           ((long long)(j % cache.block_size) * cache.n_kv_heads + g) * D + lane * DPL;
-          load_bf16<DPL>(vp, vf[u]);
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-          if (kb + kk + u < n_keys) {
-#pragma unroll
-            for (int h = 0; h < HC; ++h) {
-              if (h < nh) {
-                const float p = p_s[h][kb + kk + u];
-#pragma unroll
-                for (int i = 0; i < DPL; ++i) acc[h][i] += p * vf[u][i];
-              }
-            }
-          }
-        }
+      for (int ks = 0; ks < KS; ks += 2) {
+        const int chunk = ks * 2 + (lane >> 3);
+        uint32_t bfr[4];
+        ldmatrix_x4(k_s + krow * RB + (uint32_t)((chunk & ~7) | ((chunk ^ krow) & 7)) * 16, bfr);
+        mma_bf16_16816(sc[nt], qh[ks], bfr[0], bfr[1]);
+        mma_bf16_16816(sc[nt], ql[ks], bfr[0], bfr[1]);
+        mma_bf16_16816(sc[nt], qh[ks + 1], bfr[2], bfr[3]);
+        mma_bf16_16816(sc[nt], ql[ks + 1], bfr[2], bfr[3]);
       }
+    }
+    // mask keys past the end, row maxima over this warp's keys
+    float mx0 = -FLT_MAX, mx1 = -FLT_MAX;
 #pragma unroll
-      for (int h = 0; h < HC; ++h)
-        if (h < nh) {
+    for (int nt = 0; nt < 4; ++nt) {
+      const int key = wk0 + nt * 8 + cq;
+      if (key >= n_keys) sc[nt][0] = sc[nt][2] = -FLT_MAX;
+      if (key + 1 >= n_keys) sc[nt][1] = sc[nt][3] = -FLT_MAX;
+      mx0 = fmaxf(mx0, fmaxf(sc[nt][0], sc[nt][1]));
+      mx1 = fmaxf(mx1, fmaxf(sc[nt][2], sc[nt][3]));
+    }
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+    if ((lane & 3) == 0) {
+      wmax_s[warp][r0] = mx0;
+      wmax_s[warp][r0 + 8] = mx1;
+    }
+    if (h0 == 0) asm volatile("cp.async.wait_group 0;" ::: "memory");      // V rows have landed
+    __syncthreads();
+    mx0 = wmax_s[0][r0];
+    mx1 = wmax_s[0][r0 + 8];
 #pragma unroll
-          for (int i = 0; i < DPL; ++i) red_s[warp][h][lane * DPL + i] = acc[h][i];
-        }
+    for (int w = 1; w < NW; ++w) {
+      mx0 = fmaxf(mx0, wmax_s[w][r0]);
+      mx1 = fmaxf(mx1, wmax_s[w][r0 + 8]);
+    }
+    // ---- probabilities (A fragments, high + low) and O = P V over this warp's two 16-key steps
+    float sum0 = 0.f, sum1 = 0.f;
+    uint32_t ph[2][4], pl[2][4];
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+      const float p0 = __expf(sc[nt][0] - mx0), p1 = __expf(sc[nt][1] - mx0);     // masked scores give 0
+      const float p2 = __expf(sc[nt][2] - mx1), p3 = __expf(sc[nt][3] - mx1);
+      sum0 += p0 + p1;
+      sum1 += p2 + p3;
+      split_pair(p0, p1, ph[nt >> 1][(nt & 1) * 2], pl[nt >> 1][(nt & 1) * 2]);
+      split_pair(p2, p3, ph[nt >> 1][(nt & 1) * 2 + 1], pl[nt >> 1][(nt & 1) * 2 + 1]);
+    }
+    float oc[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) oc[nt][i] = 0.f;
+#pragma unroll
+    for (int kk = 0; kk < 2; ++kk) {
+      const int vrow = wk0 + kk * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
+#pragma unroll
+      for (int nt = 0; nt < NT; nt += 2) {
+        const int chunk = nt + (lane >> 4);
+        uint32_t bfr[4];
+        ldmatrix_x4_trans(v_s + vrow * RB + (uint32_t)((chunk & ~7) | ((chunk ^ vrow) & 7)) * 16, bfr);
+        mma_bf16_16816(oc[nt], ph[kk], bfr[0], bfr[1]);
+        mma_bf16_16816(oc[nt], pl[kk], bfr[0], bfr[1]);
+        mma_bf16_16816(oc[nt + 1], ph[kk], bfr[2], bfr[3]);
+        mma_bf16_16816(oc[nt + 1], pl[kk], bfr[2], bfr[3]);
+      }
+    }
+    sum0 += __shfl_xor_sync(0xffffffffu, sum0, 1);
+    sum0 += __shfl_xor_sync(0xffffffffu, sum0, 2);
+    sum1 += __shfl_xor_sync(0xffffffffu, sum1, 1);
+    sum1 += __shfl_xor_sync(0xffffffffu, sum1, 2);
+    if ((lane & 3) == 0) {
+      wsum_s[warp][r0] = sum0;
+      wsum_s[warp][r0 + 8] = sum1;
+    }
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      float *oa = o_red + ((long long)(warp * kPaRows + r0) * D) + nt * 8 + cq;
+      float *ob = o_red + ((long long)(warp * kPaRows + r0 + 8) * D) + nt * 8 + cq;
+      *reinterpret_cast<float2 *>(oa) = make_float2(oc[nt][0], oc[nt][1]);
+      *reinterpret_cast<float2 *>(ob) = make_float2(oc[nt][2], oc[nt][3]);
     }
     __syncthreads();
     for (int e = tid; e < nh * D; e += kPaSplitKeys) {
       const int h = e / D, c = e % D;
       float a = 0.f;
 #pragma unroll
-      for (int w = 0; w < kPaSplitKeys / 32; ++w) a += red_s[w][h][c];
+      for (int w = 0; w < NW; ++w) a += o_red[(long long)(w * kPaRows + h) * D + c];
       float *rec = partial + ((long long)(g * group + h0 + h) * n_splits + split) * (D + 2);
       rec[2 + c] = a;
       if (c == 0) {
-        rec[0] = ml_s[h][0];
-        rec[1] = ml_s[h][1];
+        float l = 0.f, m = wmax_s[0][h];
+#pragma unroll
+        for (int w = 0; w < NW; ++w) {
+          l += wsum_s[w][h];
+          m = fmaxf(m, wmax_s[w][h]);
+        }
+        rec[0] = m;
+        rec[1] = l;
       }
     }
   }
@@ -393,7 +442,7 @@ __global__ void __launch_bounds__(kPaSplitKeys) paged_attention_split_kernel(
 
 // Combines the splits of one query head: weights exp(m_s - max m) are formed once per split, then each
 // thread reduces one output dim over the splits (coalesced reads of the partial records).
-constexpr int kPaMergeMaxSplits = 1024;
+constexpr int kPaMergeMaxSplits = 2048;
 __global__ void __launch_bounds__(128) paged_attention_merge_kernel(const float *__restrict__ partial, int n_splits,
                                                                     int d, float *__restrict__ out) {
   __shared__ float w_s[kPaMergeMaxSplits];
@@ -432,10 +481,22 @@ int paged_attention(const float *q, int n_q_heads, CacheView cache, int layer, c
   if (splits > kPaMergeMaxSplits) return KV_ERR_SHAPE;   // 262,144 context tokens
   const dim3 grid(cache.n_kv_heads, splits);
   float *partial = (float *)scratch;
+  static bool attr_set[kMaxDevices] = {};
+  const int device = current_device();
+  if (device < 0) return KV_ERR_CUDA;
+  if (!attr_set[device]) {
+    KV_CUDA(cudaFuncSetAttribute(paged_attention_split_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 pa_smem_bytes(64)));
+    KV_CUDA(cudaFuncSetAttribute(paged_attention_split_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 pa_smem_bytes(128)));
+    attr_set[device] = true;
+  }
   if (cache.head_dim == 64)
-    paged_attention_split_kernel<64><<<grid, kPaSplitKeys, 0, st>>>(q, n_q_heads, cache, layer, block_table_dev, n_ctx, partial);
+    paged_attention_split_kernel<64><<<grid, kPaSplitKeys, pa_smem_bytes(64), st>>>(
+        q, n_q_heads, cache, layer, block_table_dev, n_ctx, partial);
   else if (cache.head_dim == 128)
-    paged_attention_split_kernel<128><<<grid, kPaSplitKeys, 0, st>>>(q, n_q_heads, cache, layer, block_table_dev, n_ctx, partial);
+    paged_attention_split_kernel<128><<<grid, kPaSplitKeys, pa_smem_bytes(128), st>>>(
+        q, n_q_heads, cache, layer, block_table_dev, n_ctx, partial);
   else
     return KV_ERR_SHAPE;
   KV_COUNT_LAUNCH();
