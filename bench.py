@@ -417,6 +417,18 @@ def run_ours(args):
         "t0_analog_ms": per_step["unpack"][0] + decode_ms,
         "breakdown_ms_per_step": {k: round(v[0], 4) for k, v in per_step.items()},
     }
+    # Algorithm 1 fed with the rates measured above (Section 4.2): prefill rate r_p, decode rate r_d of the
+    # source (taken as this GPU's decode step), T_0 = assembly + first decode step, on two configured links.
+    s_kv = kv.kv_bytes_per_token(shape.n_layers, shape.n_kv_heads, shape.head_dim, 2)
+    r_p, r_d = prefix / (prefill_ms * 1e-3), 1.0 / (decode_alone_ms * 1e-3)
+    t0 = (unpack_ms + decode_alone_ms) * 1e-3
+    line["window"] = {"inputs": {"k_curr": prefix, "r_p": r_p, "r_d": r_d, "s_kv": s_kv, "t0": t0, "alpha": 0.8,
+                                 "t_remain": 5.0, "t_max": 5.0, "d_t": 0.01}, "links": {}}
+    for name, goodput in (("300 Mbit/s", 300e6 / 8), ("NVLink 770 GB/s", 770e9)):
+        best, trig = kv.kv_window_select(5.0, 0.01, k_curr=float(prefix), r_p=r_p, r_d=r_d, goodput=goodput,
+                                         s_kv=float(s_kv), t0=t0, t_load=0.0, alpha=0.8, t_remain=5.0)
+        line["window"]["links"][name] = {"t_w_star": best["t_w"], "t_sit": best["t_sit"], "t_early": best["t_early"],
+                                         "trigger_now": trig}
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(synth.SHAPES[shape_name], prefix, min(prefix, args.ref_tokens),
                                             suffix_blocks=-(-suffix // synth.SHAPES[shape_name].block_size))
