@@ -1,8 +1,8 @@
 // CTA-pair variant of the projection GEMM: tcgen05.mma with cta_group::2.
 //
 // Two CTAs of a cluster (two SMs) compute one 256 x BN tile.  Each CTA loads only ITS 128 rows of A and ITS
-// half of the W tile (BN/2 rows) by TMA into its own shared memory; a single thread of the leader CTA issues
-// M=256 MMAs that read A and W from both CTAs' shared memory and accumulate rows 0-127 into the leader's TMEM
+// half of the W tile (BN/2 rows) by TMA into its own shared memory; the MMA warp of the leader CTA (converged,
+// one elected lane per instruction) issues M=256 MMAs that read A and W from both CTAs' shared memory and accumulate rows 0-127 into the leader's TMEM
 // and rows 128-255 into the peer's.  Per SM this halves the W bytes fetched from L2 and read from shared
 // memory per flop (16 KiB + 16 KiB per stage instead of 16 + 32) and leaves room for a 6-stage ring.
 // No load is shared between the CTAs: every TMA copy lands in the shared memory of the CTA that issued it;
