@@ -234,21 +234,25 @@ def test_attention_prefill_kernel(kv, torch, t, hq, hkv, d):
     assert st["max_abs"] <= MAX_ABS and st["rel_l2"] <= REL_L2, st
 
 
-def test_paged_decode_attention(kv, torch):
-    s = synth.ModelShape("pa", n_layers=2, hidden=64, n_q_heads=8, n_kv_heads=2, head_dim=128, ffn=64, vocab=16)
-    nb, n_ctx = 64, 777
-    rng = np.random.default_rng(8)
-    K = synth.bf16_round_f32(rng.standard_normal((2, n_ctx, 2, 128), dtype=np.float32))
-    V = synth.bf16_round_f32(rng.standard_normal((2, n_ctx, 2, 128), dtype=np.float32))
-    img = O.new_cache(2, nb, 16, 2, 128)
+@pytest.mark.parametrize("n_ctx,hq,hkv,d", [(777, 8, 2, 128), (1, 4, 2, 64), (128, 16, 1, 128), (129, 8, 1, 64),
+                                            (300, 40, 1, 128), (4609, 64, 8, 128)])
+def test_paged_decode_attention(kv, torch, n_ctx, hq, hkv, d):
+    """One query position against a paged context: a single key, exactly one 128-key split, one key past it, many
+    splits; groups of 2 to 40 query heads per KV head (more than the 16 rows one pass of the kernel serves)."""
+    s = synth.ModelShape("pa", n_layers=2, hidden=64, n_q_heads=hq, n_kv_heads=hkv, head_dim=d, ffn=64, vocab=16)
+    nb = -(-n_ctx // 16) + 7
+    rng = np.random.default_rng(8 + n_ctx)
+    K = synth.bf16_round_f32(rng.standard_normal((2, n_ctx, hkv, d), dtype=np.float32))
+    V = synth.bf16_round_f32(rng.standard_normal((2, n_ctx, hkv, d), dtype=np.float32))
+    img = O.new_cache(2, nb, 16, hkv, d)
     table = synth.block_permutation(9, nb)[: -(-n_ctx // 16)]
     O.write_kv(img, K, V, table)
     cache = kv.PagedCache(s, nb)
     cache.data.copy_(_bits_to_torch(torch, img.reshape(2, 2, nb, -1)))
-    q = rng.standard_normal((8, 128)).astype(np.float32)
+    q = rng.standard_normal((hq, d)).astype(np.float32)
     want = O.attention(q[None], K[1], V[1], q_pos0=n_ctx - 1)[0]
-    scratch = torch.empty(kv.kv_paged_attention_scratch_bytes(8, 128, n_ctx), dtype=torch.uint8, device="cuda")
-    out = torch.empty(8, 128, dtype=torch.float32, device="cuda")
+    scratch = torch.empty(kv.kv_paged_attention_scratch_bytes(hq, d, n_ctx), dtype=torch.uint8, device="cuda")
+    out = torch.empty(hq, d, dtype=torch.float32, device="cuda")
     kv.kv_op_paged_attention(torch.from_numpy(q).cuda(), cache, 1, torch.from_numpy(table).cuda(), n_ctx, scratch, out)
     assert np.max(np.abs(out.cpu().numpy() - want)) < 1e-4
 
