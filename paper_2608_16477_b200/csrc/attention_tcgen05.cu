@@ -50,7 +50,7 @@ __device__ long long g_attn_trace[64 * 32];
 #endif
 
 enum AttnTag { ATAG_Q = 11, ATAG_K_EMPTY = 12, ATAG_K = 13, ATAG_V = 14, ATAG_S = 15, ATAG_P = 16, ATAG_O = 17,
-               ATAG_V_EMPTY = 18, ATAG_S_FREE = 19, ATAG_PV = 20 };
+               ATAG_V_EMPTY = 18, ATAG_S_FREE = 19, ATAG_PV = 20, ATAG_QK_ISSUED = 21 };
 
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
   asm volatile(
@@ -115,8 +115,9 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
   const uint32_t smem_base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t *smem_gen = smem_raw + (smem_base - tc::smem_u32(smem_raw));
   const uint32_t bar_base = smem_base + L::kBarOff;
-  // barriers, two of each: Q full, K full, V full, K empty, V empty, S full, S free, P ready, P V done
-  enum { B_Q = 0, B_K = 1, B_V = 2, B_K_EMPTY = 3, B_V_EMPTY = 4, B_S = 5, B_S_FREE = 6, B_P = 7, B_PV = 8, B_GROUPS = 9 };
+  // barriers, two of each: Q full, K full, V full, K empty, V empty, S full, S free, P ready, P V done, Q K^T issued
+  enum { B_Q = 0, B_K = 1, B_V = 2, B_K_EMPTY = 3, B_V_EMPTY = 4, B_S = 5, B_S_FREE = 6, B_P = 7, B_PV = 8, B_QK_ISSUED = 9,
+         B_GROUPS = 10 };
   auto bar = [&](int group, int idx) { return bar_base + 8u * (group * 2 + idx); };
   uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(smem_gen + L::kBarOff + 8 * 2 * B_GROUPS);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
@@ -148,6 +149,7 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
       tc::mbar_init(bar(B_S_FREE, i), 128);
       tc::mbar_init(bar(B_P, i), 128);
       tc::mbar_init(bar(B_PV, i), 1);
+      tc::mbar_init(bar(B_QK_ISSUED, i), 1);
     }
     *abort_flag = 0;
     tc::fence_barrier_init();
@@ -229,6 +231,8 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
         }
         tc::umma_commit_warp(bar(B_S, t));
         tc::umma_commit_warp(bar(B_K_EMPTY, kst));      // second of the two arrivals frees the K stage
+        if (lane == 0) tc::mbar_arrive(bar(B_QK_ISSUED, t));   // tells the P V issuer that these MMAs are queued
+        __syncwarp();
         if (t == 0 && lane == 0) KV_ATRACE(11, j);
       }
     }
@@ -250,6 +254,12 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
         if (lane == 0) KV_ATRACE(24, j);
         for (int t = 0; t < 2 && ok; ++t) {
           ok = wwait(bar(B_P, t), j & 1, abort_flag, status, ATAG_P);
+          // The tile's softmax warps take their next scores into registers right after handing over P, and that
+          // releases the score buffer for the OTHER tile's Q K^T (key tile j + 1 for tile b, j + 2 for tile a).
+          // The tensor pipe runs MMAs in issue order and the score buffer is what both tiles wait for, so P V
+          // is queued behind that Q K^T, not in front of it.
+          const int j_qk = j + 1 + t;
+          if (ok && j_qk < n_kv) ok = wwait(bar(B_QK_ISSUED, t ^ 1), j_qk & 1, abort_flag, status, ATAG_QK_ISSUED);
           if (!ok) break;
           if (lane == 0) KV_ATRACE(8 + 2 * t, j);
           tc::tc_fence_after();
@@ -325,8 +335,8 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
         l_sum *= factor;
       }
       if (quarter == 0 && lane == 0) KV_ATRACE(t * 4 + 2, j);
-      // probabilities as packed bf16 (two keys per 32-bit column); masked scores are -inf -> 0.  The first half
-      // of the row is exponentiated before the wait for the P columns, so that the wait finds P V_{j-1} done.
+      // probabilities as packed bf16 (two keys per 32-bit column); masked scores are -inf -> 0.  The whole row is
+      // exponentiated before the wait for the P columns, so that the wait finds P V_{j-1} done.
       const float neg_m = -m_ref;
       float sum0 = 0.f, sum1 = 0.f;
       auto exps = [&](const uint32_t (&r)[32], uint32_t (&pk)[16]) {
@@ -340,9 +350,11 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
         }
       };
       auto store = [&](const uint32_t (&pk)[16], int c) { tmem_st16(p_t + c * 16, pk); };   // 32 keys
-      uint32_t pk0[16], pk1[16];
+      uint32_t pk0[16], pk1[16], pk2[16], pk3[16];
       exps(r0, pk0);
       exps(r1, pk1);
+      exps(r2, pk2);
+      exps(r3, pk3);
       // P V of the previous key tile must be done before its P columns are overwritten or O is rescaled
       if (j > 0) {
         ok = tc::mbar_wait(bar(B_PV, t), (j - 1) & 1, abort_flag, status, ATAG_PV);
@@ -364,13 +376,8 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
       }
       store(pk0, 0);
       store(pk1, 1);
-      {
-        uint32_t pk[16];
-        exps(r2, pk);
-        store(pk, 2);
-        exps(r3, pk);
-        store(pk, 3);
-      }
+      store(pk2, 2);
+      store(pk3, 3);
       l_sum += sum0 + sum1;
       tc::tmem_st_wait();
       tc::tc_fence_before();
