@@ -21,7 +21,8 @@
 // Per key tile a softmax warpgroup therefore waits only for things issued most of a step earlier (S of this
 // tile, P V of the previous one); the tensor pipe and the exponentials overlap instead of alternating.
 // TMEM columns: S [0,128)  P_a [128,192)  P_b [192,256)  O_a [256,256+D)  O_b [384,384+D).
-// Tiles are launched heaviest-first (causal work grows with the row tile index).
+// The kernel is persistent: one CTA per SM walks a list of work items (row tile, head pair), heaviest row tiles
+// first (causal work grows with the row tile index); the pipeline keeps running across items.
 // Every mbarrier wait is bounded; a wait that runs out is recorded in the status block and the CTA drains.
 #include "tc_common.cuh"
 
@@ -115,9 +116,10 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
   const uint32_t smem_base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t *smem_gen = smem_raw + (smem_base - tc::smem_u32(smem_raw));
   const uint32_t bar_base = smem_base + L::kBarOff;
-  // barriers, two of each: Q full, K full, V full, K empty, V empty, S full, S free, P ready, P V done, Q K^T issued
+  // barriers, two of each: Q full, K full, V full, K empty, V empty, S full, S free, P ready, P V done, Q K^T issued,
+  // O free (read by the epilogue), and one Q empty
   enum { B_Q = 0, B_K = 1, B_V = 2, B_K_EMPTY = 3, B_V_EMPTY = 4, B_S = 5, B_S_FREE = 6, B_P = 7, B_PV = 8, B_QK_ISSUED = 9,
-         B_GROUPS = 10 };
+         B_O_FREE = 10, B_Q_EMPTY = 11, B_GROUPS = 12 };
   auto bar = [&](int group, int idx) { return bar_base + 8u * (group * 2 + idx); };
   uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(smem_gen + L::kBarOff + 8 * 2 * B_GROUPS);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
@@ -126,17 +128,35 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
   const int group = n_q_heads / n_kv_heads;
   const int pairs = n_q_heads / 2;
   const int m_tiles = (n_tokens + kBM - 1) / kBM;
-  const int m_tile = m_tiles - 1 - (int)(blockIdx.x / pairs);     // heaviest row tiles first
-  const int pair = blockIdx.x % pairs;
-  const int head_a = 2 * pair, head_b = head_a + 1;
-  const int kv_head = head_a / group;
-  const int m0 = m_tile * kBM;                                     // first chunk row of this tile
+  const int n_items = m_tiles * pairs;
   const int n_ctx = pos0 + n_tokens;
-  // causal: key tiles up to the one holding the last row's own position
-  const int n_kv = min((n_ctx + kBN - 1) / kBN, (pos0 + m0 + kBM - 1) / kBN + 1);
-  const int q_col[2] = {head_a * D, head_b * D};
-  const int k_col = (n_q_heads + kv_head) * D;
-  const int v_col = (n_q_heads + n_kv_heads + kv_head) * D;
+  // Work items (row tile, head pair), heaviest row tiles first.
+  // Every role walks the same list and keeps running counters, so the pipeline never drains between items: the
+  // loads and the first Q K^T of the next item run under the last step and the epilogue of this one.
+  // The k-th item of this CTA: rounds of gridDim.x items, walked forwards in even rounds and backwards in odd ones,
+  // so that the CTA with the heaviest item of one round gets the lightest of the next (the list is sorted).
+  auto item_of = [&](int k) {
+    const int base = k * (int)gridDim.x;
+    return base + ((k & 1) ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)blockIdx.x);
+  };
+  struct Item {
+    int m0, n_kv, head_a, q_col0, q_col1, k_col, v_col;
+  };
+  auto get_item = [&](int it) {
+    Item w;
+    const int m_tile = m_tiles - 1 - it / pairs;
+    const int pair = it % pairs;
+    w.head_a = 2 * pair;
+    const int kv_head = w.head_a / group;
+    w.m0 = m_tile * kBM;                                    // first chunk row of this tile
+    // causal: key tiles up to the one holding the last row's own position
+    w.n_kv = min((n_ctx + kBN - 1) / kBN, (pos0 + w.m0 + kBM - 1) / kBN + 1);
+    w.q_col0 = w.head_a * D;
+    w.q_col1 = w.q_col0 + D;
+    w.k_col = (n_q_heads + kv_head) * D;
+    w.v_col = (n_q_heads + n_kv_heads + kv_head) * D;
+    return w;
+  };
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
@@ -150,7 +170,9 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
       tc::mbar_init(bar(B_P, i), 128);
       tc::mbar_init(bar(B_PV, i), 1);
       tc::mbar_init(bar(B_QK_ISSUED, i), 1);
+      tc::mbar_init(bar(B_O_FREE, i), 128);
     }
+    tc::mbar_init(bar(B_Q_EMPTY, 0), 2);       // one arrival per Q K^T issuer, after its last MMA of an item
     *abort_flag = 0;
     tc::fence_barrier_init();
   }
@@ -167,35 +189,45 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
     if (lane == 0) {
       tc::tma_prefetch_desc(&tma_qkv);
-      for (int t = 0; t < 2; ++t) {
-        tc::mbar_expect_tx(bar(B_Q, t), L::kTileBytes);
-        for (int a = 0; a < kAtoms; ++a)
-          tc::tma_load_2d(smem_base + L::kQOff + t * L::kTileBytes + a * kBoxBytes, &tma_qkv, q_col[t] + a * 64, pos0 + m0,
-                          bar(B_Q, t));
-      }
-      auto load_k = [&](int j) {
-        const int st = j % kKS;
-        if (!tc::mbar_wait(bar(B_K_EMPTY, st), ((j / kKS) & 1) ^ 1, abort_flag, status, ATAG_K_EMPTY)) return false;
-        const uint32_t k_s = smem_base + L::kKOff + st * L::kTileBytes;
-        tc::mbar_expect_tx(bar(B_K, st), L::kTileBytes);
-        for (int a = 0; a < kAtoms; ++a)
-          tc::tma_load_2d(k_s + a * kBoxBytes, &tma_qkv, k_col + a * 64, j * kBN, bar(B_K, st));
-        return true;
-      };
-      auto load_v = [&](int j) {
-        const int st = j % kVS;
-        if (!tc::mbar_wait(bar(B_V_EMPTY, st), ((j / kVS) & 1) ^ 1, abort_flag, status, ATAG_V_EMPTY)) return false;
-        const uint32_t v_s = smem_base + L::kVOff + st * L::kTileBytes;
-        tc::mbar_expect_tx(bar(B_V, st), L::kTileBytes);
-        for (int a = 0; a < kAtoms; ++a)
-          tc::tma_load_2d(v_s + a * kBoxBytes, &tma_qkv, v_col + a * 64, j * kBN, bar(B_V, st));
-        return true;
-      };
-      // in the order the tiles are consumed: K_0, then K_{j+1} before V_j
-      bool ok = load_k(0);
-      for (int j = 0; j < n_kv && ok; ++j) {
-        if (j + 1 < n_kv) ok = load_k(j + 1);
-        if (ok) ok = load_v(j);
+      int lk = 0, lv = 0;                       // K and V tiles loaded so far (ring positions)
+      bool ok = true;
+      for (int k = 0, it = item_of(0); it < n_items && ok; it = item_of(++k)) {
+        const Item w = get_item(it);
+        auto load_k = [&](int j) {
+          const int st = lk % kKS;
+          if (!tc::mbar_wait(bar(B_K_EMPTY, st), ((lk / kKS) & 1) ^ 1, abort_flag, status, ATAG_K_EMPTY)) return false;
+          const uint32_t k_s = smem_base + L::kKOff + st * L::kTileBytes;
+          tc::mbar_expect_tx(bar(B_K, st), L::kTileBytes);
+          for (int a = 0; a < kAtoms; ++a)
+            tc::tma_load_2d(k_s + a * kBoxBytes, &tma_qkv, w.k_col + a * 64, j * kBN, bar(B_K, st));
+          ++lk;
+          return true;
+        };
+        auto load_v = [&](int j) {
+          const int st = lv % kVS;
+          if (!tc::mbar_wait(bar(B_V_EMPTY, st), ((lv / kVS) & 1) ^ 1, abort_flag, status, ATAG_V_EMPTY)) return false;
+          const uint32_t v_s = smem_base + L::kVOff + st * L::kTileBytes;
+          tc::mbar_expect_tx(bar(B_V, st), L::kTileBytes);
+          for (int a = 0; a < kAtoms; ++a)
+            tc::tma_load_2d(v_s + a * kBoxBytes, &tma_qkv, w.v_col + a * 64, j * kBN, bar(B_V, st));
+          ++lv;
+          return true;
+        };
+        // the Q tiles may be replaced once the last Q K^T of the previous item has run
+        ok = tc::mbar_wait(bar(B_Q_EMPTY, 0), (k & 1) ^ 1, abort_flag, status, ATAG_Q);
+        if (!ok) break;
+        for (int t = 0; t < 2; ++t) {
+          tc::mbar_expect_tx(bar(B_Q, t), L::kTileBytes);
+          for (int a = 0; a < kAtoms; ++a)
+            tc::tma_load_2d(smem_base + L::kQOff + t * L::kTileBytes + a * kBoxBytes, &tma_qkv,
+                            (t == 0 ? w.q_col0 : w.q_col1) + a * 64, pos0 + w.m0, bar(B_Q, t));
+        }
+        // in the order the tiles are consumed: K_0, then K_{j+1} before V_j
+        ok = load_k(0);
+        for (int j = 0; j < w.n_kv && ok; ++j) {
+          if (j + 1 < w.n_kv) ok = load_k(j + 1);
+          if (ok) ok = load_v(j);
+        }
       }
     }
   } else if (warp == 1 || warp == 2) {
@@ -213,27 +245,31 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
       const uint32_t s_tmem = tmem_base + kTmemS;
       const int t = warp - 1;
       const uint32_t q_s = smem_base + L::kQOff + t * L::kTileBytes;
-      // The score buffer is used in the order a_0 b_0 a_1 b_1 ...: each use starts once the previous user
-      // (the other tile) has taken its scores into registers (S free).
-      bool ok = wwait(bar(B_Q, t), 0, abort_flag, status, ATAG_Q);
-      for (int j = 0; j < n_kv && ok; ++j) {
-        const int kst = j % kKS;
-        ok = wwait(bar(B_K, kst), (j / kKS) & 1, abort_flag, status, ATAG_K);
-        if (ok && j + t > 0) ok = wwait(bar(B_S_FREE, t ^ 1), (t == 0 ? j - 1 : j) & 1, abort_flag, status, ATAG_S_FREE);
-        if (!ok) break;
-        tc::tc_fence_after();
-        if (t == 0 && lane == 0) KV_ATRACE(9, j);
-        const uint32_t k_s = smem_base + L::kKOff + kst * L::kTileBytes;
+      // The score buffer is used in the order a_0 b_0 a_1 b_1 ... (across items too): each use starts once the
+      // previous user (the other tile) has taken its scores into registers (S free).
+      int s = 0;                                // key-tile steps so far, over all items
+      bool ok = true;
+      for (int k = 0, it = item_of(0); it < n_items && ok; it = item_of(++k)) {
+        const int n_kv = get_item(it).n_kv;
+        ok = wwait(bar(B_Q, t), k & 1, abort_flag, status, ATAG_Q);
+        for (int j = 0; j < n_kv && ok; ++j, ++s) {
+          const int kst = s % kKS;
+          ok = wwait(bar(B_K, kst), (s / kKS) & 1, abort_flag, status, ATAG_K);
+          if (ok && s + t > 0) ok = wwait(bar(B_S_FREE, t ^ 1), (t == 0 ? s - 1 : s) & 1, abort_flag, status, ATAG_S_FREE);
+          if (!ok) break;
+          tc::tc_fence_after();
+          const uint32_t k_s = smem_base + L::kKOff + kst * L::kTileBytes;
 #pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks) {
-          const uint32_t off = (ks / 4) * kBoxBytes + (ks % 4) * 32;
-          tc::umma_bf16_warp(s_tmem, tc::umma_desc_k128(q_s + off), tc::umma_desc_k128(k_s + off), idesc_qk, ks != 0);
+          for (int ks = 0; ks < D / 16; ++ks) {
+            const uint32_t off = (ks / 4) * kBoxBytes + (ks % 4) * 32;
+            tc::umma_bf16_warp(s_tmem, tc::umma_desc_k128(q_s + off), tc::umma_desc_k128(k_s + off), idesc_qk, ks != 0);
+          }
+          tc::umma_commit_warp(bar(B_S, t));
+          tc::umma_commit_warp(bar(B_K_EMPTY, kst));      // second of the two arrivals frees the K stage
+          if (j == n_kv - 1) tc::umma_commit_warp(bar(B_Q_EMPTY, 0));
+          if (lane == 0) tc::mbar_arrive(bar(B_QK_ISSUED, t));   // tells the P V issuer that these MMAs are queued
+          __syncwarp();
         }
-        tc::umma_commit_warp(bar(B_S, t));
-        tc::umma_commit_warp(bar(B_K_EMPTY, kst));      // second of the two arrivals frees the K stage
-        if (lane == 0) tc::mbar_arrive(bar(B_QK_ISSUED, t));   // tells the P V issuer that these MMAs are queued
-        __syncwarp();
-        if (t == 0 && lane == 0) KV_ATRACE(11, j);
       }
     }
   } else if (warp == 3) {
@@ -246,32 +282,35 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
       constexpr uint32_t idesc_pv = tc::umma_idesc_bf16(kBM, D) | (1u << 16);   // B (= V) is MN-major
       const uint32_t p_tmem[2] = {tmem_base + kTmemP0, tmem_base + kTmemP1};
       const uint32_t o_tmem[2] = {tmem_base + kTmemO0, tmem_base + kTmemO1};
+      int s = 0;
       bool ok = true;
-      for (int j = 0; j < n_kv && ok; ++j) {
-        const int vst = j % kVS;
-        ok = wwait(bar(B_V, vst), (j / kVS) & 1, abort_flag, status, ATAG_V);
-        const uint32_t v_s = smem_base + L::kVOff + vst * L::kTileBytes;
-        if (lane == 0) KV_ATRACE(24, j);
-        for (int t = 0; t < 2 && ok; ++t) {
-          ok = wwait(bar(B_P, t), j & 1, abort_flag, status, ATAG_P);
-          // The tile's softmax warps take their next scores into registers right after handing over P, and that
-          // releases the score buffer for the OTHER tile's Q K^T (key tile j + 1 for tile b, j + 2 for tile a).
-          // The tensor pipe runs MMAs in issue order and the score buffer is what both tiles wait for, so P V
-          // is queued behind that Q K^T, not in front of it.
-          const int j_qk = j + 1 + t;
-          if (ok && j_qk < n_kv) ok = wwait(bar(B_QK_ISSUED, t ^ 1), j_qk & 1, abort_flag, status, ATAG_QK_ISSUED);
-          if (!ok) break;
-          if (lane == 0) KV_ATRACE(8 + 2 * t, j);
-          tc::tc_fence_after();
+      for (int k = 0, it = item_of(0); it < n_items && ok; it = item_of(++k)) {
+        const int n_kv = get_item(it).n_kv;
+        for (int j = 0; j < n_kv && ok; ++j, ++s) {
+          const int vst = s % kVS;
+          ok = wwait(bar(B_V, vst), (s / kVS) & 1, abort_flag, status, ATAG_V);
+          const uint32_t v_s = smem_base + L::kVOff + vst * L::kTileBytes;
+          for (int t = 0; t < 2 && ok; ++t) {
+            ok = wwait(bar(B_P, t), s & 1, abort_flag, status, ATAG_P);
+            // The tile's softmax warps take their next scores into registers right after handing over P, and that
+            // releases the score buffer for the OTHER tile's Q K^T (key tile j + 1 for tile b, j + 2 for tile a).
+            // The tensor pipe runs MMAs in issue order and the score buffer is what both tiles wait for, so P V
+            // is queued behind that Q K^T, not in front of it (inside an item; at its end P V must not wait).
+            const int j_qk = j + 1 + t;
+            if (ok && j_qk < n_kv) ok = wwait(bar(B_QK_ISSUED, t ^ 1), (s + 1 + t) & 1, abort_flag, status, ATAG_QK_ISSUED);
+            // the first P V of an item overwrites O: the epilogue of the previous item must have read it
+            if (ok && j == 0) ok = wwait(bar(B_O_FREE, t), (k & 1) ^ 1, abort_flag, status, ATAG_O);
+            if (!ok) break;
+            tc::tc_fence_after();
 #pragma unroll
-          for (int ks = 0; ks < kBN / 16; ++ks)   // 16 keys per slice: 8 TMEM columns of P, 2048 bytes of V
-            tc::umma_bf16_ts_warp(o_tmem[t], p_tmem[t] + ks * 8, umma_desc_mn128(v_s + ks * 2048, kBoxBytes), idesc_pv,
-                             (j | ks) != 0);
-          tc::umma_commit_warp(bar(B_PV, t));
-          if (lane == 0) KV_ATRACE(25 + t, j);
+            for (int ks = 0; ks < kBN / 16; ++ks)   // 16 keys per slice: 8 TMEM columns of P, 2048 bytes of V
+              tc::umma_bf16_ts_warp(o_tmem[t], p_tmem[t] + ks * 8, umma_desc_mn128(v_s + ks * 2048, kBoxBytes), idesc_pv,
+                                    (j | ks) != 0);
+            tc::umma_commit_warp(bar(B_PV, t));
+          }
+          if (!ok) break;
+          tc::umma_commit_warp(bar(B_V_EMPTY, vst));
         }
-        if (!ok) break;
-        tc::umma_commit_warp(bar(B_V_EMPTY, vst));
       }
     }
   } else {
@@ -280,134 +319,139 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
     const int t = (warp - 4) >> 2;                 // 0: tile a, 1: tile b
     const int quarter = warp & 3;
     const int row_in_tile = quarter * 32 + lane;
-    const int qi = pos0 + m0 + row_in_tile;        // absolute query position
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
     const uint32_t s_t = tmem_base + lane_base + kTmemS;
     const uint32_t p_t = tmem_base + lane_base + (t == 0 ? kTmemP0 : kTmemP1);
     const uint32_t o_t = tmem_base + lane_base + (t == 0 ? kTmemO0 : kTmemO1);
-    float m_ref = -INFINITY, l_sum = 0.f;
+    int s = 0;                                     // key-tile steps so far, over all items
     bool ok = true;
-    for (int j = 0; j < n_kv; ++j) {
-      ok = tc::mbar_wait(bar(B_S, t), j & 1, abort_flag, status, ATAG_S);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      if (quarter == 0 && lane == 0) KV_ATRACE(t * 4 + 0, j);
-      tc::tc_fence_after();
-      const bool diag = (j * kBN + kBN - 1 > pos0 + m0);   // tile reaches past the first row's position
-      const int limit = qi - j * kBN;              // keys with column > limit are masked
-      // the whole row of S (128 fp32) in registers: four loads in flight, one wait; then S may be overwritten
-      uint32_t r0[32], r1[32], r2[32], r3[32];
-      tc::tmem_ld32(s_t + 0, r0);
-      tc::tmem_ld32(s_t + 32, r1);
-      tc::tmem_ld32(s_t + 64, r2);
-      tc::tmem_ld32(s_t + 96, r3);
-      tc::tmem_ld_wait();
-      tc::tc_fence_before();
-      tc::mbar_arrive(bar(B_S_FREE, t));
-      if (quarter == 0 && lane == 0) KV_ATRACE(t * 4 + 1, j);
-      float mx = -INFINITY;
-      if (!diag) {
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          mx = fmaxf(mx, fmaxf(fmaxf(__uint_as_float(r0[i]), __uint_as_float(r1[i])),
-                               fmaxf(__uint_as_float(r2[i]), __uint_as_float(r3[i]))));
-        }
-      } else {
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          if (i > limit) r0[i] = 0xff800000u;        // -inf
-          if (32 + i > limit) r1[i] = 0xff800000u;
-          if (64 + i > limit) r2[i] = 0xff800000u;
-          if (96 + i > limit) r3[i] = 0xff800000u;
-          mx = fmaxf(mx, fmaxf(fmaxf(__uint_as_float(r0[i]), __uint_as_float(r1[i])),
-                               fmaxf(__uint_as_float(r2[i]), __uint_as_float(r3[i]))));
-        }
-      }
-      mx *= scale_log2;
-      bool rescale = false;
-      float factor = 1.f;
-      if (j == 0) {
-        m_ref = mx;
-      } else if (mx > m_ref + kRescaleThreshold) {
-        rescale = true;
-        factor = exp2f(m_ref - mx);
-        m_ref = mx;
-        l_sum *= factor;
-      }
-      if (quarter == 0 && lane == 0) KV_ATRACE(t * 4 + 2, j);
-      // probabilities as packed bf16 (two keys per 32-bit column); masked scores are -inf -> 0.  The whole row is
-      // exponentiated before the wait for the P columns, so that the wait finds P V_{j-1} done.
-      const float neg_m = -m_ref;
-      float sum0 = 0.f, sum1 = 0.f;
-      auto exps = [&](const uint32_t (&r)[32], uint32_t (&pk)[16]) {
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const float p0 = exp2f(fmaf(__uint_as_float(r[2 * i]), scale_log2, neg_m));
-          const float p1 = exp2f(fmaf(__uint_as_float(r[2 * i + 1]), scale_log2, neg_m));
-          sum0 += p0;
-          sum1 += p1;
-          pk[i] = pack2(p0, p1);
-        }
-      };
-      auto store = [&](const uint32_t (&pk)[16], int c) { tmem_st16(p_t + c * 16, pk); };   // 32 keys
-      uint32_t pk0[16], pk1[16], pk2[16], pk3[16];
-      exps(r0, pk0);
-      exps(r1, pk1);
-      exps(r2, pk2);
-      exps(r3, pk3);
-      // P V of the previous key tile must be done before its P columns are overwritten or O is rescaled
-      if (j > 0) {
-        ok = tc::mbar_wait(bar(B_PV, t), (j - 1) & 1, abort_flag, status, ATAG_PV);
+    for (int k = 0, it = item_of(0); it < n_items && ok; it = item_of(++k)) {
+      const Item w = get_item(it);
+      const int m0 = w.m0, n_kv = w.n_kv;
+      const int qi = pos0 + m0 + row_in_tile;      // absolute query position
+      float m_ref = -INFINITY, l_sum = 0.f;
+      for (int j = 0; j < n_kv; ++j, ++s) {
+        ok = tc::mbar_wait(bar(B_S, t), s & 1, abort_flag, status, ATAG_S);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
+        if (quarter == 0 && lane == 0) KV_ATRACE(t * 4 + 0, s);
         tc::tc_fence_after();
-      }
-      if (quarter == 0 && lane == 0) KV_ATRACE(12 + t, j);
-      if (__any_sync(0xffffffffu, rescale)) {
-#pragma unroll 1
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t r[32];
-          tc::tmem_ld32(o_t + c * 32, r);
-          tc::tmem_ld_wait();
-#pragma unroll
-          for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * factor);
-          tmem_st32(o_t + c * 32, r);
-        }
-      }
-      store(pk0, 0);
-      store(pk1, 1);
-      store(pk2, 2);
-      store(pk3, 3);
-      l_sum += sum0 + sum1;
-      tc::tmem_st_wait();
-      tc::tc_fence_before();
-      tc::mbar_arrive(bar(B_P, t));
-      if (quarter == 0 && lane == 0) KV_ATRACE(t * 4 + 3, j);
-      if (lane == 0) KV_ATRACE(16 + t * 4 + quarter, j);
-    }
-    if (ok) {
-      ok = tc::mbar_wait(bar(B_PV, t), (n_kv - 1) & 1, abort_flag, status, ATAG_O);
-      ok = __all_sync(0xffffffffu, ok);
-    }
-    if (ok) {
-      tc::tc_fence_after();
-      const float inv = 1.f / l_sum;
-      const int head = (t == 0) ? head_a : head_b;
-      const int out_row = m0 + row_in_tile;        // row inside the chunk
-      bf16 *orow = out + (long long)out_row * n_q_heads * D + head * D;
-#pragma unroll 1
-      for (int c = 0; c < D / 32; ++c) {
-        uint32_t r[32];
-        tc::tmem_ld32(o_t + c * 32, r);
+        const bool diag = (j * kBN + kBN - 1 > pos0 + m0);   // tile reaches past the first row's position
+        const int limit = qi - j * kBN;              // keys with column > limit are masked
+        // the whole row of S (128 fp32) in registers: four loads in flight, one wait; then S may be overwritten
+        uint32_t r0[32], r1[32], r2[32], r3[32];
+        tc::tmem_ld32(s_t + 0, r0);
+        tc::tmem_ld32(s_t + 32, r1);
+        tc::tmem_ld32(s_t + 64, r2);
+        tc::tmem_ld32(s_t + 96, r3);
         tc::tmem_ld_wait();
-        if (out_row < n_tokens) {
+        tc::tc_fence_before();
+        tc::mbar_arrive(bar(B_S_FREE, t));
+        float mx = -INFINITY;
+        if (!diag) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            mx = fmaxf(mx, fmaxf(fmaxf(__uint_as_float(r0[i]), __uint_as_float(r1[i])),
+                                 fmaxf(__uint_as_float(r2[i]), __uint_as_float(r3[i]))));
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            if (i > limit) r0[i] = 0xff800000u;        // -inf
+            if (32 + i > limit) r1[i] = 0xff800000u;
+            if (64 + i > limit) r2[i] = 0xff800000u;
+            if (96 + i > limit) r3[i] = 0xff800000u;
+            mx = fmaxf(mx, fmaxf(fmaxf(__uint_as_float(r0[i]), __uint_as_float(r1[i])),
+                                 fmaxf(__uint_as_float(r2[i]), __uint_as_float(r3[i]))));
+          }
+        }
+        mx *= scale_log2;
+        bool rescale = false;
+        float factor = 1.f;
+        if (j == 0) {
+          m_ref = mx;
+        } else if (mx > m_ref + kRescaleThreshold) {
+          rescale = true;
+          factor = exp2f(m_ref - mx);
+          m_ref = mx;
+          l_sum *= factor;
+        }
+        // probabilities as packed bf16 (two keys per 32-bit column); masked scores are -inf -> 0.  The whole row is
+        // exponentiated before the wait for the P columns, so that the wait finds P V_{j-1} done.
+        const float neg_m = -m_ref;
+        float sum0 = 0.f, sum1 = 0.f;
+        auto exps = [&](const uint32_t (&r)[32], uint32_t (&pk)[16]) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float p0 = exp2f(fmaf(__uint_as_float(r[2 * i]), scale_log2, neg_m));
+            const float p1 = exp2f(fmaf(__uint_as_float(r[2 * i + 1]), scale_log2, neg_m));
+            sum0 += p0;
+            sum1 += p1;
+            pk[i] = pack2(p0, p1);
+          }
+        };
+        auto store = [&](const uint32_t (&pk)[16], int c) { tmem_st16(p_t + c * 16, pk); };   // 32 keys
+        uint32_t pk0[16], pk1[16], pk2[16], pk3[16];
+        exps(r0, pk0);
+        exps(r1, pk1);
+        exps(r2, pk2);
+        exps(r3, pk3);
+        // P V of the previous key tile must be done before its P columns are overwritten or O is rescaled (for the
+        // first key tile of an item the epilogue of the previous item has already waited for it)
+        if (j > 0) {
+          ok = tc::mbar_wait(bar(B_PV, t), (s - 1) & 1, abort_flag, status, ATAG_PV);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          tc::tc_fence_after();
+        }
+        if (__any_sync(0xffffffffu, rescale)) {
+#pragma unroll 1
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t r[32];
+            tc::tmem_ld32(o_t + c * 32, r);
+            tc::tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * factor);
+            tmem_st32(o_t + c * 32, r);
+          }
+        }
+        store(pk0, 0);
+        store(pk1, 1);
+        store(pk2, 2);
+        store(pk3, 3);
+        l_sum += sum0 + sum1;
+        tc::tmem_st_wait();
+        tc::tc_fence_before();
+        tc::mbar_arrive(bar(B_P, t));
+        if (quarter == 0 && lane == 0) KV_ATRACE(t * 4 + 3, s);
+      }
+      if (!ok) break;
+      // ---- epilogue of the item: O / l -> bf16 rows.  O is taken into registers in one go and handed back, so
+      // the next item's first P V does not wait for the stores.
+      ok = tc::mbar_wait(bar(B_PV, t), (s - 1) & 1, abort_flag, status, ATAG_O);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc::tc_fence_after();
+      uint32_t o_r[D / 32][32];
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) tc::tmem_ld32(o_t + c * 32, o_r[c]);
+      tc::tmem_ld_wait();
+      tc::tc_fence_before();
+      tc::mbar_arrive(bar(B_O_FREE, t));
+      const float inv = 1.f / l_sum;
+      const int head = w.head_a + t;
+      const int out_row = m0 + row_in_tile;        // row inside the chunk
+      if (out_row < n_tokens) {
+        bf16 *orow = out + (long long)out_row * n_q_heads * D + head * D;
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
           uint4 *dst = reinterpret_cast<uint4 *>(orow + c * 32);
 #pragma unroll
           for (int v = 0; v < 4; ++v)
-            dst[v] = make_uint4(pack2(__uint_as_float(r[8 * v]) * inv, __uint_as_float(r[8 * v + 1]) * inv),
-                                pack2(__uint_as_float(r[8 * v + 2]) * inv, __uint_as_float(r[8 * v + 3]) * inv),
-                                pack2(__uint_as_float(r[8 * v + 4]) * inv, __uint_as_float(r[8 * v + 5]) * inv),
-                                pack2(__uint_as_float(r[8 * v + 6]) * inv, __uint_as_float(r[8 * v + 7]) * inv));
+            dst[v] = make_uint4(pack2(__uint_as_float(o_r[c][8 * v]) * inv, __uint_as_float(o_r[c][8 * v + 1]) * inv),
+                                pack2(__uint_as_float(o_r[c][8 * v + 2]) * inv, __uint_as_float(o_r[c][8 * v + 3]) * inv),
+                                pack2(__uint_as_float(o_r[c][8 * v + 4]) * inv, __uint_as_float(o_r[c][8 * v + 5]) * inv),
+                                pack2(__uint_as_float(o_r[c][8 * v + 6]) * inv, __uint_as_float(o_r[c][8 * v + 7]) * inv));
         }
       }
     }
@@ -486,7 +530,9 @@ int attention_prefill_tc(const bf16 *qkv_ctx, int n_tokens, int pos0, int n_q_he
   }
   if (regs_ok_dev[device] != 1) return KV_ERR_SHAPE;
   const int m_tiles = (n_tokens + kBM - 1) / kBM;
-  const int grid = m_tiles * (n_q_heads / 2);
+  const int items = m_tiles * (n_q_heads / 2);
+  const int sms = sm_count(device);
+  const int grid = items < sms ? items : sms;      // persistent: one CTA per SM walks the items
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)head_dim);
   DeviceStatus *status = reinterpret_cast<DeviceStatus *>(status_dev);
   if (head_dim == 64)
