@@ -2,10 +2,10 @@
 // The qkv buffer holds one row per context position: rows [0, pos0) carry the K/V of an already cached
 // prefix (gathered from its pages), rows [pos0, pos0 + T) the chunk's post-RoPE Q, K and V.
 //
-// One CTA works on ONE 128-row query tile of TWO query heads that share a KV head (tiles "a" and "b"), so
+// A work item is ONE 128-row query tile of TWO query heads that share a KV head (tiles "a" and "b"), so
 // every K/V tile fetched by TMA feeds both.
 //
-//   warp 0      TMA producer of Q (once) and of the K and V tiles (128 keys each).
+//   warp 0      TMA producer of Q (once per item) and of the K and V tiles (128 keys each).
 //   warps 1, 2  S = Q K^T of tile a and of tile b (both operands K-major in shared memory); warp 1 also
 //               allocates TMEM.  The whole warp runs the loop, one elected lane issues each tcgen05.mma.
 //   warp 3      O += P V of both tiles (P read from TMEM, V as an MN-major shared-memory operand: no
