@@ -216,8 +216,11 @@ def test_rmsnorm_rows(kv, torch):
     assert np.all(np.abs(got - want) <= 2.0 ** -8 * np.abs(want) + 1e-6)
 
 
+# the last two cases give the persistent kernel more work items than SMs: 200 items (a partial second round,
+# walked backwards) and 300 items (two full rounds and a partial third) on 148 SMs
 @pytest.mark.parametrize("t,hq,hkv,d", [(70, 4, 2, 64), (200, 8, 1, 128), (129, 2, 2, 128), (1000, 4, 2, 128),
-                                      (384, 8, 2, 64), (128, 2, 1, 128), (1, 2, 1, 64)])
+                                      (384, 8, 2, 64), (128, 2, 1, 128), (1, 2, 1, 64), (6400, 8, 2, 64),
+                                      (3200, 24, 4, 64)])
 def test_attention_prefill_kernel(kv, torch, t, hq, hkv, d):
     rng = np.random.default_rng(7 + t)
     qkv = synth.bf16_round_f32(rng.standard_normal((t, (hq + 2 * hkv) * d), dtype=np.float32))
