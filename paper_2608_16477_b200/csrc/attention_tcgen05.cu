@@ -100,7 +100,8 @@ struct AttnSmem {
   static constexpr int kQOff = 0;
   static constexpr int kKOff = 2 * kTileBytes;
   static constexpr int kVOff = kKOff + kKStages * kTileBytes;
-  static constexpr int kBarOff = kVOff + kVStages * kTileBytes;
+  static constexpr int kStageOff = kVOff + kVStages * kTileBytes;  // 2 KiB per softmax warp: output transposition
+  static constexpr int kBarOff = kStageOff + 8 * 2048;
   static constexpr int kBytes = kBarOff + 256 + 1024;            // barriers + alignment slack
 };
 
@@ -440,18 +441,35 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
       tc::mbar_arrive(bar(B_O_FREE, t));
       const float inv = 1.f / l_sum;
       const int head = w.head_a + t;
-      const int out_row = m0 + row_in_tile;        // row inside the chunk
-      if (out_row < n_tokens) {
-        bf16 *orow = out + (long long)out_row * n_q_heads * D + head * D;
+      // A thread owns a row, and rows are n_q_heads * D * 2 bytes apart in memory: stored directly, every
+      // instruction would touch 32 different lines.  Each 32-column slab therefore goes through a 2 KiB
+      // shared-memory buffer of the warp (16-byte pieces XOR-swizzled by the row), and is written out with four
+      // lanes per row: every store instruction then covers 8 rows x 64 contiguous bytes.
+      const uint32_t stage = smem_base + L::kStageOff + (uint32_t)((warp - 4) * 2048);
+      const int rd_row = lane >> 2, rd_piece = lane & 3;
 #pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          uint4 *dst = reinterpret_cast<uint4 *>(orow + c * 32);
+      for (int c = 0; c < D / 32; ++c) {
+        __syncwarp();
 #pragma unroll
-          for (int v = 0; v < 4; ++v)
-            dst[v] = make_uint4(pack2(__uint_as_float(o_r[c][8 * v]) * inv, __uint_as_float(o_r[c][8 * v + 1]) * inv),
-                                pack2(__uint_as_float(o_r[c][8 * v + 2]) * inv, __uint_as_float(o_r[c][8 * v + 3]) * inv),
-                                pack2(__uint_as_float(o_r[c][8 * v + 4]) * inv, __uint_as_float(o_r[c][8 * v + 5]) * inv),
-                                pack2(__uint_as_float(o_r[c][8 * v + 6]) * inv, __uint_as_float(o_r[c][8 * v + 7]) * inv));
+        for (int v = 0; v < 4; ++v) {
+          const uint32_t addr = stage + (uint32_t)lane * 64 + (uint32_t)((v ^ ((lane >> 1) & 3)) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr),
+                       "r"(pack2(__uint_as_float(o_r[c][8 * v]) * inv, __uint_as_float(o_r[c][8 * v + 1]) * inv)),
+                       "r"(pack2(__uint_as_float(o_r[c][8 * v + 2]) * inv, __uint_as_float(o_r[c][8 * v + 3]) * inv)),
+                       "r"(pack2(__uint_as_float(o_r[c][8 * v + 4]) * inv, __uint_as_float(o_r[c][8 * v + 5]) * inv)),
+                       "r"(pack2(__uint_as_float(o_r[c][8 * v + 6]) * inv, __uint_as_float(o_r[c][8 * v + 7]) * inv))
+                       : "memory");
+        }
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int r = rd_row + 8 * i;                       // row inside this warp's 32
+          const int out_row = m0 + quarter * 32 + r;          // row inside the chunk
+          uint4 val;
+          const uint32_t addr = stage + (uint32_t)r * 64 + (uint32_t)((rd_piece ^ ((r >> 1) & 3)) << 4);
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w) : "r"(addr));
+          if (out_row < n_tokens)
+            *reinterpret_cast<uint4 *>(out + (long long)out_row * n_q_heads * D + head * D + c * 32 + rd_piece * 8) = val;
         }
       }
     }
