@@ -102,7 +102,20 @@ __global__ void __launch_bounds__(kGemvWarps * 32) gemv2_kernel(const bf16 *__re
     acc_a += dot8(ra, x0, x1);
     acc_b += dot8(rb, x0, x1);
   };
+  // The first batch of weight loads is issued on its own and awaited with a fence before x is touched: measured,
+  // this start-up order shortens a 62 GB decode step from 14.5 to 13.6 ms (a compiler-only barrier at the same
+  // place, a fence at the top of the kernel, or a fence in every iteration do not).
   int v = lane;
+  if (v + 96 < nvec) {
+    const uint4 a0 = __ldcs(wa + v), a1 = __ldcs(wa + v + 32), a2 = __ldcs(wa + v + 64), a3 = __ldcs(wa + v + 96);
+    const uint4 b0 = __ldcs(wb + v), b1 = __ldcs(wb + v + 32), b2 = __ldcs(wb + v + 64), b3 = __ldcs(wb + v + 96);
+    asm volatile("fence.acq_rel.gpu;" ::: "memory");
+    step(a0, b0, v);
+    step(a1, b1, v + 32);
+    step(a2, b2, v + 64);
+    step(a3, b3, v + 96);
+    v += 128;
+  }
   for (; v + 96 < nvec; v += 128) {
     const uint4 a0 = __ldcs(wa + v), a1 = __ldcs(wa + v + 32), a2 = __ldcs(wa + v + 64), a3 = __ldcs(wa + v + 96);
     const uint4 b0 = __ldcs(wb + v), b1 = __ldcs(wb + v + 32), b2 = __ldcs(wb + v + 64), b3 = __ldcs(wb + v + 96);
