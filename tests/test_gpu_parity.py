@@ -153,7 +153,7 @@ def test_gemm_tensor_core(kv, torch, m, n, k, mode):
         assert np.max(np.abs(got - want)) <= tol, error_stats(got, want)
 
 
-@pytest.mark.parametrize("m,n,k", [(256, 256, 64), (300, 520, 192), (1000, 1048, 512), (4096, 5120, 256)])
+@pytest.mark.parametrize("m,n,k", [(129, 520, 192), (256, 256, 64), (300, 520, 192), (1000, 1048, 512), (4096, 5120, 256)])
 @pytest.mark.parametrize("mode", [0, 1, 2])
 def test_gemm_cta_pair_identical_to_single_cta(kv, torch, m, n, k, mode):
     """The cta_group::2 kernel (two SMs per 256-row tile) accumulates in the same order as the one-CTA kernel."""
