@@ -384,6 +384,7 @@ int prefill_layers(kv_model *m, const CacheView &cv, PrefillWs &w, int total_row
       ProfScope ps(PROF_GEMM_QKV, st);
       QkvRopeArgs qa;
       qa.rope = w.rope;
+      qa.rope_rows = t;
       qa.block_table = w.table;
       qa.row_pos = row_pos;
       qa.row_block = row_block;

@@ -76,7 +76,9 @@ enum GemmMode { GEMM_STORE_BF16 = 0, GEMM_RESID_F32 = 1, GEMM_SWIGLU = 2, GEMM_Q
 
 // Extra arguments of the fused QKV epilogue: RoPE on the accumulators, K/V stored into the paged cache.
 struct QkvRopeArgs {
-  const float2 *rope;       // [n_tokens, head_dim/2] (cos, sin) of each row's position
+  const float2 *rope;       // [head_dim/2, rope_rows] (cos, sin) of each row's position: the 32 rows of a warp read
+                            // consecutive entries
+  int rope_rows;            // rows of that table (tokens of the call)
   const int *block_table;   // device; single request: row r is position pos0 + r of this table
   const int *row_pos;       // batched requests (else nullptr): position of each row inside its request
   const int *row_block;     // batched requests: physical block that holds each row

@@ -104,18 +104,18 @@ int rmsnorm_rows(const float *x, const bf16 *gain, int rows, int dim, float eps,
   return KV_OK;
 }
 
-// table[t, j] = (cos, sin)(pos * base^(-2j/d)), angle formed in fp64 so that positions in the
+// table[j, t] = (cos, sin)(pos_t * base^(-2j/d)) (frequency-major), angle formed in fp64 so that positions in the
 // tens of thousands keep full fp32 accuracy after the final rounding.
 __global__ void rope_table_kernel(float2 *table, int pos0, int n_tokens, int half, float base,
                                   const int *__restrict__ row_pos) {
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= n_tokens * half) return;
-  const int t = idx / half, j = idx - t * half;
+  const int j = idx / n_tokens, t = idx - j * n_tokens;      // consecutive threads: consecutive tokens of one frequency
   const double theta = pow((double)base, -(double)j / (double)half);
   double s, c;
   const int pos = row_pos != nullptr ? row_pos[t] : pos0 + t;
   sincos((double)pos * theta, &s, &c);
-  table[idx] = make_float2((float)c, (float)s);
+  table[(long long)j * n_tokens + t] = make_float2((float)c, (float)s);
 }
 
 int rope_table(float2 *table, int pos0, int n_tokens, int head_dim, float base, cudaStream_t st, const int *row_pos) {

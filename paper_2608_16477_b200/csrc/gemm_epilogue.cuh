@@ -42,7 +42,7 @@ __device__ __forceinline__ void gemm_epilogue_slab(uint32_t t_row, int row, int 
       block = qa.row_block != nullptr ? qa.row_block[row] : qa.block_table[pos / qa.cache.block_size];
       slot_off = (long long)(pos % qa.cache.block_size) * qa.cache.n_kv_heads * d;
     }
-    const float2 *cs_row = qa.rope + (long long)row * half;
+    const float2 *cs_row = qa.rope + (live ? row : 0);      // entry j of this row: cs_row[j * rope_rows]
     bf16 *orow = out + (long long)row * n;
 #pragma unroll 1
     for (int c = 0; c < BN / 32; ++c) {
@@ -59,7 +59,7 @@ __device__ __forceinline__ void gemm_epilogue_slab(uint32_t t_row, int row, int 
           float a[32], b[32];
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
-            const float2 cs = cs_row[j0 + i];
+            const float2 cs = cs_row[(long long)(j0 + i) * qa.rope_rows];
             const float x = __uint_as_float(lo[i]), y = __uint_as_float(hi[i]);
             a[i] = x * cs.x - y * cs.y;
             b[i] = y * cs.x + x * cs.y;
