@@ -247,13 +247,13 @@ int32_t kv_op_paged_attention(const float *q_dev, int32_t n_q_heads, const kv_ca
  * inside the library, which every GPU that loads the library keeps until exit.
  *  - Limit: kv_paged_attention_scratch_bytes(n_q_heads, head_dim, n_ctx) must not exceed
  *    KV_NOALLOC_SCRATCH_BYTES, otherwise KV_ERR_WORKSPACE is returned and nothing is launched
- *    (64 query heads of dimension 128 fit up to 8,064 context tokens).
+ *    (64 query heads of dimension 128 fit up to 16,128 context tokens).
  *  - The call never allocates or frees memory.  Its first call on a device looks up the array's device
  *    address (once per device); make that first call before starting any stream capture.
  *  - All calls on a device share the one array and it keeps whatever the last call left there.  A call
  *    writes every partial it later reads, so stale contents are harmless, but two calls whose kernels can
  *    overlap on the GPU (different streams) race on it: serialise them. */
-#define KV_NOALLOC_SCRATCH_BYTES (2 * 1024 * 1024)
+#define KV_NOALLOC_SCRATCH_BYTES (4 * 1024 * 1024)
 int32_t kv_op_paged_attention_noalloc(const float *q_dev, int32_t n_q_heads, const kv_cache_desc *cache,
                                       int32_t layer, const int32_t *block_table_dev, int32_t n_ctx,
                                       float *out_dev, void *stream);

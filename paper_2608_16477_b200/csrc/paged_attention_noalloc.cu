@@ -12,7 +12,7 @@
 
 namespace {
 
-// 2 MiB of split-KV partials (m, l, acc[head_dim] per query head and key split).  Every GPU that loads
+// 4 MiB of split-KV partials (m, l, acc[head_dim] per query head and key split).  Every GPU that loads
 // the library holds this array until the process exits.
 constexpr long long kNoAllocScratchBytes = KV_NOALLOC_SCRATCH_BYTES;
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];

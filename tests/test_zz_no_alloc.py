@@ -47,9 +47,9 @@ def test_noalloc_rejects_contexts_beyond_its_array():
     q = torch.zeros(64, 128, device="cuda")
     out = torch.zeros(64, 128, device="cuda")
     table = torch.zeros(8, dtype=torch.int32, device="cuda")
-    too_long = 8064 + 1               # one 128-key split beyond what 2 MiB of partials can hold for 64 heads of 128
-    assert kv.kv_paged_attention_scratch_bytes(64, 128, 8064) <= 2 * 1024 * 1024
-    assert kv.kv_paged_attention_scratch_bytes(64, 128, too_long) > 2 * 1024 * 1024
+    too_long = 16128 + 1              # one 128-key split beyond what 4 MiB of partials can hold for 64 heads of 128
+    assert kv.kv_paged_attention_scratch_bytes(64, 128, 16128) <= 4 * 1024 * 1024
+    assert kv.kv_paged_attention_scratch_bytes(64, 128, too_long) > 4 * 1024 * 1024
     with pytest.raises(kv.KVError) as e:
         kv.kv_op_paged_attention_noalloc(q, cache, 0, table, too_long, out)
     assert e.value.status == -10      # KV_ERR_WORKSPACE: nothing was launched
