@@ -1,7 +1,7 @@
 """Runs ONE kernel of the hot path a few times at the benchmark's shapes, for profiler captures.
 
   python -m paper_2608_16477_b200.profile_case gemm_gate_up [--tokens 4096] [--iters 3]
-  cases: gemm_qkv, gemm_o, gemm_gate_up, gemm_down, attention, pack, unpack, decode_gemv, decode_attention
+  cases: gemm_qkv, gemm_o, gemm_gate_up, gemm_down, attention, pack, unpack, decode_gemv, decode_attention, prefill_layer
 
 Inputs are synthetic and larger than L2 where the kernel is bandwidth-bound; a few GB at most are held on
 the device so a multi-pass capture stays short.  Prints the CUDA-event time per launch.
@@ -91,6 +91,24 @@ def main():
             state["i"] += 1
             kv.kv_op_gemv(ws[state["i"] % 4], x, 2, y, gain=gain, eps=1e-6)
         work, unit = ws[0].numel() * 2 / 1e9, "GB/s"
+    elif a.case == "prefill_layer":
+        # one decoder layer of the shape through kv_prefill_prefix (logits on, so the layer is not truncated after
+        # its QKV projection): the way to capture the QKV + RoPE + paged-store GEMM, whose epilogue needs a cache
+        s1 = s.with_layers(1)
+        mat = lambda r, c: rnd(r, c, std=0.02)
+        ones = lambda: torch.ones(s.hidden, dtype=torch.bfloat16, device=dev)
+        layer = lambda l: {"attn_norm": ones(), "ffn_norm": ones(), "w_qkv": mat(s.qkv_dim, s.hidden),
+                           "w_o": mat(s.hidden, s.q_dim), "w_gate_up": mat(2 * s.ffn, s.hidden), "w_down": mat(s.hidden, s.ffn)}
+        head = {"embed": mat(s.vocab, s.hidden), "lm_head": mat(s.vocab, s.hidden), "final_norm": ones()}
+        model = kv.Model(s1, head, layer)
+        cache = kv.PagedCache(s1, t // s.block_size + 1)
+        ids = synth.token_ids(s1, 0, t)
+        table = synth.block_permutation(1, t // s.block_size + 1)[: t // s.block_size]
+        ws = model.workspace(kv.KV_OP_PREFILL, t)
+        logits = torch.empty(s.vocab, dtype=torch.float32, device=dev)
+        run = lambda: kv.kv_prefill_prefix(model, cache, ids, table, logits_out=logits, workspace=ws)
+        lin = 2.0 * t * (s.hidden * s.qkv_dim + s.q_dim * s.hidden + 3 * s.hidden * s.ffn)
+        work, unit = (lin + 2.0 * s.n_q_heads * s.head_dim * t * (t + 1)) / 1e12, "TFLOP/s"
     elif a.case == "decode_attention":
         # one layer's paged attention of a decode step at context a.tokens + 512 (the bench's resume position),
         # rotating over 4 layers of a fragmented cache so consecutive launches read cold pages
