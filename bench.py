@@ -207,6 +207,23 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------ our arm
+def build_model(kv, torch, shape, seed=1000):
+    """Random-init weights of the shape, N(0, init_std^2) in bf16, norm gains 1, created on the device."""
+    gen = torch.Generator(device="cuda").manual_seed(seed)
+
+    def mat(rows, cols):
+        return torch.empty(rows, cols, dtype=torch.bfloat16, device="cuda").normal_(0.0, shape.init_std, generator=gen)
+
+    def layer(l):
+        ones = torch.ones(shape.hidden, dtype=torch.bfloat16, device="cuda")
+        return {"attn_norm": ones, "ffn_norm": ones.clone(), "w_qkv": mat(shape.qkv_dim, shape.hidden),
+                "w_o": mat(shape.hidden, shape.q_dim), "w_gate_up": mat(2 * shape.ffn, shape.hidden),
+                "w_down": mat(shape.hidden, shape.ffn)}
+    head = {"embed": mat(shape.vocab, shape.hidden), "lm_head": mat(shape.vocab, shape.hidden),
+            "final_norm": torch.ones(shape.hidden, dtype=torch.bfloat16, device="cuda")}
+    return kv.Model(shape, head, layer), gen
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -230,19 +247,7 @@ def run_ours(args):
     bs = shape.block_size
     n = prefix + suffix
     seed = 1000 + rank
-    gen = torch.Generator(device="cuda").manual_seed(seed)
-
-    def mat(rows, cols):
-        return torch.empty(rows, cols, dtype=torch.bfloat16, device="cuda").normal_(0.0, shape.init_std, generator=gen)
-
-    def layer(l):
-        ones = torch.ones(shape.hidden, dtype=torch.bfloat16, device="cuda")
-        return {"attn_norm": ones, "ffn_norm": ones.clone(), "w_qkv": mat(shape.qkv_dim, shape.hidden),
-                "w_o": mat(shape.hidden, shape.q_dim), "w_gate_up": mat(2 * shape.ffn, shape.hidden),
-                "w_down": mat(shape.hidden, shape.ffn)}
-    head = {"embed": mat(shape.vocab, shape.hidden), "lm_head": mat(shape.vocab, shape.hidden),
-            "final_norm": torch.ones(shape.hidden, dtype=torch.bfloat16, device="cuda")}
-    model = kv.Model(shape, head, layer)
+    model, gen = build_model(kv, torch, shape, seed)
 
     ids = synth.token_ids(shape, seed, n + 1)
     src = kv.PagedCache(shape, pool_blocks)
@@ -455,6 +460,64 @@ def stress_geometry(kv, torch, shape):
     return counts, total, src_blocks, dst_blocks, block_bytes
 
 
+def run_stream_overlap(args):
+    """Source-side incremental suffix synchronisation (Section 4.3): decode steps of the 32B shape with every completed
+    suffix block packed on a side stream and delivered to a receiver on the same GPU, against the same steps alone."""
+    import torch
+    import paper_2608_16477_b200 as kv
+    from paper_2608_16477_b200 import streaming
+    kv.load()
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    shape = synth.SHAPES["32b"]
+    k_split, n_steps = 4096, 64
+    bs = shape.block_size
+    nb = (k_split + n_steps) // bs + 1
+    model, _ = build_model(kv, torch, shape)
+    src = kv.PagedCache(shape, nb + 8)
+    tgt = kv.PagedCache(shape, nb + 8)
+    kv.kv_fill_pattern(src.data, src.data.numel() * 2, seed=5)
+    src.data.bitwise_and_(0x3FFF)                      # finite bf16 content standing in for the prefix K/V
+    table = synth.block_permutation(1, nb + 8)[:nb]
+    ids = synth.token_ids(shape, 0, k_split + n_steps + 1)
+    logits = torch.empty(shape.vocab, dtype=torch.float32, device="cuda")
+    ws = model.workspace(kv.KV_OP_DECODE, k_split + n_steps + 1)
+    stream = torch.cuda.current_stream()
+
+    def decode_run(streamer):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for pos in range(k_split, k_split + n_steps):
+            kv.kv_decode_step(model, src, int(ids[pos]), pos, table[: pos // bs + 1], logits, workspace=ws)
+            if streamer is not None:
+                streamer.on_token(pos)
+                streamer.pump()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n_steps
+
+    for _ in range(max(args.warmup, 3)):
+        decode_run(None)
+    plain = min(decode_run(None) for _ in range(args.steps))
+    times, sent = [], 0
+    for rep in range(args.steps):
+        rx = streaming.SuffixReceiver(tgt, 1, rep, k_split, n_steps // bs + 1, list(range(nb + 8))[-(n_steps // bs + 1):])
+        st = streaming.SuffixStreamer(src, table, k_split, 1, rep, streaming.LoopbackTransport(rx))
+        times.append(decode_run(st))
+        sent = len(st.sent)
+    overlapped = min(times)
+    block_bytes = shape.n_layers * 2 * src.page_bytes
+    line = {"metric": "decode_ms_with_suffix_streaming", "value": overlapped, "unit": "ms", "n_gpus": 1, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": overlapped, "higher_is_better": False, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "stream-overlap", "shape": "32b", "k_split": k_split, "decode_steps": n_steps,
+                       "blocks_streamed": sent, "block_bytes": block_bytes},
+            "decode_ms_alone": plain, "decode_ms_streaming": overlapped, "slowdown": overlapped / plain - 1.0,
+            "gpu_launches": int(kv.kv_launch_count())}
+    print(json.dumps(line))
+    return 0
+
+
 def run_pack_stress(args):
     import torch
     import paper_2608_16477_b200 as kv
@@ -516,7 +579,7 @@ def main():
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="32b-4k", choices=sorted(WORKLOADS) + ["pack-stress"])
+    ap.add_argument("--workload", default="32b-4k", choices=sorted(WORKLOADS) + ["pack-stress", "stream-overlap"])
     ap.add_argument("--layers", type=int, default=0, help="debug: reduced depth (invalid as a bench number)")
     ap.add_argument("--ref-tokens", type=int, default=2048, help="prefix tokens in the oracle's bounded sample")
     ap.add_argument("--ref-warmup", type=int, default=0)
@@ -525,6 +588,8 @@ def main():
     args.warmup_given = any(a == "--warmup" or a.startswith("--warmup=") for a in sys.argv[1:])
     if args.workload == "pack-stress" and args.impl != "reference":
         return run_pack_stress(args)
+    if args.workload == "stream-overlap" and args.impl != "reference":
+        return run_stream_overlap(args)
     if args.impl == "reference":
         return run_reference(args)
     return run_ours(args)
