@@ -518,6 +518,51 @@ def run_stream_overlap(args):
     return 0
 
 
+def run_batched_prefill(args):
+    """Concurrent migrations (Section 4.5): K prefixes rebuilt by one kv_prefill_prefix_batched call against K separate
+    kv_prefill_prefix calls, 32B shape."""
+    import torch
+    import paper_2608_16477_b200 as kv
+    kv.load()
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    shape = synth.SHAPES["32b"]
+    k_req, n = 4, 512
+    model, _ = build_model(kv, torch, shape)
+    blocks_each = n // shape.block_size
+    cache = kv.PagedCache(shape, k_req * blocks_each + 8, fill=0)
+    perm = synth.block_permutation(3, k_req * blocks_each + 8)
+    ids = [synth.token_ids(shape, 10 + i, n) for i in range(k_req)]
+    tabs = [perm[i * blocks_each:(i + 1) * blocks_each].copy() for i in range(k_req)]
+
+    def separate():
+        for i in range(k_req):
+            kv.kv_prefill_prefix(model, cache, ids[i], tabs[i])
+
+    def batched():
+        kv.kv_prefill_prefix_batched(model, cache, ids, tabs)
+
+    def timed(fn):
+        for _ in range(max(args.warmup, 3)):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / args.steps
+    ms_sep, ms_bat = timed(separate), timed(batched)
+    line = {"metric": METRIC, "value": k_req * n / (ms_bat * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_bat, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "batched-prefill", "shape": "32b", "requests": k_req, "prefix_tokens": n},
+            "batched_ms": ms_bat, "separate_calls_ms": ms_sep,
+            "separate_calls_tokens_per_s": k_req * n / (ms_sep * 1e-3), "gpu_launches": int(kv.kv_launch_count())}
+    print(json.dumps(line))
+    return 0
+
+
 def run_pack_stress(args):
     import torch
     import paper_2608_16477_b200 as kv
@@ -579,7 +624,7 @@ def main():
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="32b-4k", choices=sorted(WORKLOADS) + ["pack-stress", "stream-overlap"])
+    ap.add_argument("--workload", default="32b-4k", choices=sorted(WORKLOADS) + ["pack-stress", "stream-overlap", "batched-prefill"])
     ap.add_argument("--layers", type=int, default=0, help="debug: reduced depth (invalid as a bench number)")
     ap.add_argument("--ref-tokens", type=int, default=2048, help="prefix tokens in the oracle's bounded sample")
     ap.add_argument("--ref-warmup", type=int, default=0)
@@ -590,6 +635,8 @@ def main():
         return run_pack_stress(args)
     if args.workload == "stream-overlap" and args.impl != "reference":
         return run_stream_overlap(args)
+    if args.workload == "batched-prefill" and args.impl != "reference":
+        return run_batched_prefill(args)
     if args.impl == "reference":
         return run_reference(args)
     return run_ours(args)
