@@ -4,6 +4,9 @@ unpack/assemble and the resumed decode step, through the C ABI.
 
   python bench.py --gpus N --steps K --warmup W            (N > 1: launched by torch.distributed.run)
   python bench.py --impl reference ...                     (the CPU oracle on a bounded sample)
+  python bench.py --workload pack-stress | stream-overlap | batched-prefill
+                                                           (side measurements: copy steady state, suffix streaming
+                                                            under decode, concurrent migrations; one GPU)
 
 One "step" is one pass of the whole path for one request of the workload.  Every rank runs an independent
 replica (the path does not shard: no data-path collective), so scaling is weak and `value` is the sum of
