@@ -238,7 +238,7 @@ def test_attention_prefill_kernel(kv, torch, t, hq, hkv, d):
 
 
 @pytest.mark.parametrize("n_ctx,hq,hkv,d", [(777, 8, 2, 128), (1, 4, 2, 64), (128, 16, 1, 128), (129, 8, 1, 64),
-                                            (300, 40, 1, 128), (4609, 64, 8, 128)])
+                                            (300, 40, 1, 128), (4609, 64, 8, 128), (20011, 8, 1, 128)])
 def test_paged_decode_attention(kv, torch, n_ctx, hq, hkv, d):
     """One query position against a paged context: a single key, exactly one 128-key split, one key past it, many
     splits; groups of 2 to 40 query heads per KV head (more than the 16 rows one pass of the kernel serves)."""
