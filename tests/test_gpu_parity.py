@@ -237,6 +237,26 @@ def test_attention_prefill_kernel(kv, torch, t, hq, hkv, d):
     assert st["max_abs"] <= MAX_ABS and st["rel_l2"] <= REL_L2, st
 
 
+def test_attention_prefill_long_context_sampled_rows(kv, torch):
+    """8,192 tokens (64 key tiles for the last row tile, 256 work items on 148 SMs): three windows of query rows are
+    checked against the oracle, which scores each window against the keys up to its last row."""
+    t, hq, hkv, d = 8192, 8, 2, 128
+    rng = np.random.default_rng(99)
+    qkv = synth.bf16_round_f32(rng.standard_normal((t, (hq + 2 * hkv) * d), dtype=np.float32))
+    out = torch.empty(t, hq * d, dtype=torch.bfloat16, device="cuda")
+    status = torch.zeros(64, dtype=torch.int32, device="cuda")
+    kv.kv_op_attention_prefill(torch.from_numpy(qkv).cuda().to(torch.bfloat16), hq, hkv, d, out, status=status)
+    assert int(status[0]) == 0
+    got = out.float().cpu().numpy().reshape(t, hq, d)
+    q = qkv[:, : hq * d].reshape(t, hq, d)
+    k = qkv[:, hq * d: (hq + hkv) * d].reshape(t, hkv, d)
+    v = qkv[:, (hq + hkv) * d:].reshape(t, hkv, d)
+    for r0, r1 in ((0, 130), (4030, 4170), (8060, 8192)):
+        want = O.attention(q[r0:r1], k[:r1], v[:r1], q_pos0=r0)
+        st = error_stats(got[r0:r1], want)
+        assert st["max_abs"] <= MAX_ABS and st["rel_l2"] <= REL_L2, (r0, st)
+
+
 @pytest.mark.parametrize("n_ctx,hq,hkv,d", [(777, 8, 2, 128), (1, 4, 2, 64), (128, 16, 1, 128), (129, 8, 1, 64),
                                             (300, 40, 1, 128), (4609, 64, 8, 128), (20011, 8, 1, 128)])
 def test_paged_decode_attention(kv, torch, n_ctx, hq, hkv, d):
