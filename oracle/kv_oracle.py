@@ -23,8 +23,10 @@ It shares no code with the CUDA path and never imports it.
 
 Pins (tests/test_oracle_pins.py): Eq. (1) closed form and the 262,144 B/token footnote,
 RMSNorm/SwiGLU closed forms, RoPE invariants, brute-force loop attention on tiny inputs,
-torch SDPA as a black-box library cross-check, causality between the full-sequence and the
-incremental code paths, pack/unpack by a five-deep byte loop.
+torch SDPA as a black-box library cross-check, causality between the full-sequence, the
+chunk-by-chunk (cached-prefix) and the incremental code paths, the fp32 library matmul against
+the fp64 one and against an error bound, the bf16 storage points against the library cast at
+each of them, pack/unpack by a five-deep byte loop.
 Parity unpinned: fidelity to real Qwen3/Llama checkpoints (no weights are available).
 """
 from __future__ import annotations
@@ -218,6 +220,38 @@ def forward_full(shape, head: dict, layers, token_ids, mm_dtype=np.float64,
         if not all_logits:
             logits = logits[0]
     return np.stack(ks), np.stack(vs), logits
+
+
+def forward_chunked(shape, head: dict, layers, token_ids, chunk_sizes, mm_dtype=np.float64,
+                    want_logits: bool = True, act_bf16: bool = False):
+    """The same forward evaluated chunk by chunk (continued prefill, Section 4.5: the migration prefill is
+    split into chunks that interleave with resident decoding).  Chunk c covers the next chunk_sizes[c] tokens;
+    its rows attend to the K/V that earlier chunks left (k_past / v_past of `layer_forward`) and to
+    themselves.  Returns (K, V, logits) like `forward_full`; logits are those of the last row of the last
+    chunk.  `layers` is called once per (chunk, layer).
+    """
+    token_ids = np.asarray(token_ids)
+    assert sum(chunk_sizes) == len(token_ids) and all(c > 0 for c in chunk_sizes)
+    emb = np.asarray(head["embed"], dtype=np.float64)
+    k_done = [np.zeros((0, shape.n_kv_heads, shape.head_dim)) for _ in range(shape.n_layers)]
+    v_done = [np.zeros((0, shape.n_kv_heads, shape.head_dim)) for _ in range(shape.n_layers)]
+    p0 = 0
+    x = None
+    for ci, c in enumerate(chunk_sizes):
+        pos = np.arange(p0, p0 + c)
+        x = emb[token_ids[p0:p0 + c]]
+        final_chunk = ci == len(chunk_sizes) - 1
+        for l in range(shape.n_layers):
+            stop = final_chunk and (l == shape.n_layers - 1) and not want_logits
+            x, k, v = layer_forward(shape, layers(l), x, pos, k_past=k_done[l], v_past=v_done[l],
+                                    mm_dtype=mm_dtype, skip_after_kv=stop, act_bf16=act_bf16)
+            k_done[l] = np.concatenate([k_done[l], k], axis=0)
+            v_done[l] = np.concatenate([v_done[l], v], axis=0)
+        p0 += c
+    logits = None
+    if want_logits:
+        logits = _mm(rmsnorm(x[-1:], head["final_norm"], shape.rms_eps), head["lm_head"], mm_dtype)[0]
+    return np.stack(k_done), np.stack(v_done), logits
 
 
 def decode_step(shape, head: dict, layers, token_id: int, pos: int, k_cache, v_cache):

@@ -7,7 +7,7 @@ Plain Python floats (fp64), each function one equation of the paper in its notat
 Readings where the paper is silent: candidates are {0, dT, 2 dT, ...} up to and including T_limit when it is a
 multiple of dT (no extra candidate at T_limit otherwise); ties of J go to the smallest window; the smoothing
 factor of the moving average is a parameter (new = beta * sample + (1 - beta) * old).
-Pinned by closed forms and special cases in tests/test_window_model.py.
+Pinned by closed forms and special cases in tests/test_window_oracle.py.
 """
 from __future__ import annotations
 

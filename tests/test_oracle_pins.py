@@ -397,3 +397,134 @@ def test_bf16_storage_points_only_round():
     a = O.layer_forward(t, w, x, np.array([0]), skip_after_kv=True)
     b = O.layer_forward(t, w, x, np.array([0]), skip_after_kv=True, act_bf16=True)
     assert np.array_equal(a[1], b[1]) and np.array_equal(a[2], b[2])
+
+
+# ---------------------------------------------------------------- continued (chunked) prefill
+@pytest.mark.parametrize("name", ["tiny", "tiny-sharp"])
+@pytest.mark.parametrize("chunks", [(16,) * 6, (48, 48), (33, 1, 47, 15), (96,)])
+def test_chunked_prefill_equals_full(name, chunks):
+    """Chunk-by-chunk evaluation over a cached prefix (k_past / v_past) is the same function as the
+    single-pass forward: every chunk size, ragged splits and a one-token chunk included."""
+    s = synth.SHAPES[name]
+    head = synth.head_weights(s, 0)
+    lw = [synth.layer_weights(s, 0, l) for l in range(s.n_layers)]
+    ids = synth.token_ids(s, 0, sum(chunks))
+    Kf, Vf, lf = O.forward_full(s, head, lambda l: lw[l], ids)
+    Kc, Vc, lc = O.forward_chunked(s, head, lambda l: lw[l], ids, chunks)
+    for got, want in ((Kc, Kf), (Vc, Vf), (lc, lf)):
+        assert got.shape == want.shape
+        assert np.max(np.abs(got - want)) <= 1e-10 * np.max(np.abs(want))
+    # K/V-only form: the last layer of the last chunk stops after its K/V, same values
+    Kn, Vn, ln = O.forward_chunked(s, head, lambda l: lw[l], ids, chunks, want_logits=False)
+    assert ln is None and np.array_equal(Kn, Kc) and np.array_equal(Vn, Vc)
+
+
+def test_chunked_prefill_past_is_used_and_ordered():
+    """A wrong past must show: dropping the cached prefix, or pairing its keys with the wrong values, changes the
+    chunk's output (reordering keys and values together does not: every past position is visible to every
+    row of the chunk, and the positions are already rotated into the keys)."""
+    s = synth.SHAPES["tiny-sharp"]
+    w = synth.layer_weights(s, 0, 0)
+    r = np.random.default_rng(3)
+    x = r.standard_normal((40, s.hidden))
+    xa, ka, va = O.layer_forward(s, w, x[:24], np.arange(24))
+    xb, kb, vb = O.layer_forward(s, w, x[24:], np.arange(24, 40), k_past=ka, v_past=va)
+    xf, kf, vf = O.layer_forward(s, w, x, np.arange(40))
+    assert np.allclose(np.concatenate([xa, xb]), xf, rtol=0, atol=1e-11 * np.max(np.abs(xf)))
+    assert np.allclose(np.concatenate([ka, kb]), kf, rtol=0, atol=1e-12)
+    x_nopast, _, _ = O.layer_forward(s, w, x[24:], np.arange(24, 40))
+    x_rev, _, _ = O.layer_forward(s, w, x[24:], np.arange(24, 40), k_past=ka[::-1], v_past=va[::-1])
+    x_mix, _, _ = O.layer_forward(s, w, x[24:], np.arange(24, 40), k_past=ka[::-1], v_past=va)
+    assert np.max(np.abs(x_nopast - xb)) > 1e-3 and np.max(np.abs(x_mix - xb)) > 1e-3
+    assert np.max(np.abs(x_rev - xb)) <= 1e-11 * np.max(np.abs(xb))
+    # K and V of the new rows never depend on the past
+    _, k2, v2 = O.layer_forward(s, w, x[24:], np.arange(24, 40), skip_after_kv=True)
+    assert np.array_equal(k2, kb) and np.array_equal(v2, vb)
+
+
+# ---------------------------------------------------------------- fp32 library matmul (used on the largest shapes)
+def test_fp32_matmul_against_fp64_and_error_bound():
+    r = np.random.default_rng(8)
+    x = synth.bf16_round_f32(r.standard_normal((256, 384), dtype=np.float32))
+    w = synth.bf16_round_f32(r.standard_normal((512, 384), dtype=np.float32) * np.float32(0.05))
+    exact = O._mm(x, w, np.float64)
+    got = O._mm(x, w, np.float32)
+    assert got.dtype == np.float64 and got.shape == (256, 512)
+    assert np.sqrt(np.sum((got - exact) ** 2) / np.sum(exact ** 2)) <= 1e-5
+    # textbook bound for a length-k fp32 dot product in any summation order: |err| <= k u sum|x||w| (u = 2^-24),
+    # plus the final rounding of the result
+    k, u = 384, 2.0 ** -24
+    bound = (k + 1) * u * (np.abs(x).astype(np.float64) @ np.abs(w).astype(np.float64).T)
+    assert np.all(np.abs(got - exact) <= bound)
+    # orientation: y = x W^T
+    assert np.array_equal(O._mm(np.eye(3), np.arange(6.0).reshape(2, 3), np.float32), np.arange(6.0).reshape(2, 3).T)
+
+
+def test_fp32_matmul_forward_tracks_fp64_forward():
+    s = synth.SHAPES["tiny-sharp"]
+    head = synth.head_weights(s, 0)
+    lw = [synth.layer_weights(s, 0, l) for l in range(s.n_layers)]
+    ids = synth.token_ids(s, 0, 64)
+    K0, V0, l0 = O.forward_full(s, head, lambda l: lw[l], ids)
+    K1, V1, l1 = O.forward_full(s, head, lambda l: lw[l], ids, mm_dtype=np.float32)
+    for a, b in ((K1, K0), (V1, V0), (l1, l0)):
+        assert np.sqrt(np.sum((a - b) ** 2) / np.sum(b ** 2)) <= 1e-5
+
+
+# ---------------------------------------------------------------- bf16 storage points, one by one
+def test_bf16_storage_points_against_library_casts():
+    """Where the storage-precision evaluation rounds: one layer restated with library tensor ops in fp64 and a
+    library bfloat16 cast at each of the tensors a 16-bit pipeline keeps between contractions (normed input,
+    post-RoPE Q and K, V, attention output, normed FFN input, SwiGLU output) and nowhere else (the residual
+    stream, scores, probabilities and accumulators stay wide)."""
+    torch = pytest.importorskip("torch")
+    F = torch.nn.functional
+    s = synth.SHAPES["tiny-sharp"]
+    w = synth.layer_weights(s, 0, 1)
+    r = np.random.default_rng(12)
+    t = 24
+    x = r.standard_normal((t, s.hidden)) * 1.7
+    pos = np.arange(5, 5 + t)
+    kp = synth.bf16_round_f32(r.standard_normal((5, s.n_kv_heads, s.head_dim), dtype=np.float32))
+    vp = synth.bf16_round_f32(r.standard_normal((5, s.n_kv_heads, s.head_dim), dtype=np.float32))
+    got_x, got_k, got_v = O.layer_forward(s, w, x, pos, k_past=kp, v_past=vp, act_bf16=True)
+
+    def cast(a):
+        return a.to(torch.bfloat16).to(torch.float64)
+
+    def norm(a, g):
+        return a * torch.rsqrt((a * a).mean(-1, keepdim=True) + s.rms_eps) * g
+
+    def rot(a):     # [T, H, d]
+        half = s.head_dim // 2
+        inv = torch.tensor([s.rope_base ** (-2.0 * j / s.head_dim) for j in range(half)], dtype=torch.float64)
+        ang = torch.tensor(pos, dtype=torch.float64)[:, None] * inv[None]
+        c, sn = torch.cos(ang)[:, None], torch.sin(ang)[:, None]
+        a1, a2 = a[..., :half], a[..., half:]
+        return torch.cat([a1 * c - a2 * sn, a2 * c + a1 * sn], -1)
+
+    W = {k: torch.tensor(np.asarray(v), dtype=torch.float64) for k, v in w.items()}
+    xt = torch.tensor(x)
+    h = cast(norm(xt, W["attn_norm"]))
+    qkv = h @ W["w_qkv"].T
+    hq, hkv, d = s.n_q_heads, s.n_kv_heads, s.head_dim
+    q = cast(rot(qkv[:, : hq * d].reshape(t, hq, d)))
+    k = cast(rot(qkv[:, hq * d: (hq + hkv) * d].reshape(t, hkv, d)))
+    v = cast(qkv[:, (hq + hkv) * d:].reshape(t, hkv, d))
+    k_all = torch.cat([torch.tensor(kp, dtype=torch.float64), k]).repeat_interleave(hq // hkv, dim=1)
+    v_all = torch.cat([torch.tensor(vp, dtype=torch.float64), v]).repeat_interleave(hq // hkv, dim=1)
+    mask = torch.arange(5 + t)[None, :] <= torch.tensor(pos)[:, None]
+    o = F.scaled_dot_product_attention(q.permute(1, 0, 2)[None], k_all.permute(1, 0, 2)[None],
+                                       v_all.permute(1, 0, 2)[None], attn_mask=mask)[0].permute(1, 0, 2)
+    x1 = xt + cast(o).reshape(t, hq * d) @ W["w_o"].T
+    h2 = cast(norm(x1, W["ffn_norm"]))
+    ab = h2 @ W["w_gate_up"].T
+    m = cast(F.silu(ab[:, : s.ffn]) * ab[:, s.ffn:])
+    x2 = x1 + m @ W["w_down"].T
+    assert np.array_equal(got_k, k.numpy()) or np.max(np.abs(got_k - k.numpy())) <= 2.0 ** -7 * np.max(np.abs(got_k))
+    # identical rounding decisions except where a pre-rounding value sits within fp64 noise of a tie
+    assert np.mean(got_k != k.numpy()) < 1e-3 and np.mean(got_v != v.numpy()) < 1e-3
+    assert np.max(np.abs(got_x - x2.numpy())) <= 1e-9 * np.max(np.abs(got_x))
+    # and the roundings matter: the exact layer differs by far more than the agreement above
+    ex_x, _, _ = O.layer_forward(s, w, x, pos, k_past=kp, v_past=vp)
+    assert np.max(np.abs(ex_x - got_x)) > 1e-4
