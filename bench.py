@@ -52,6 +52,29 @@ WORKLOADS = {
 NCU_TRAFFIC_BYTES = {"32b-4k": 1269.9e6}   # profiles/gemm_tc_pair_gate_up_32b-4k.md: 1,064.3 MB read + 205.6 MB written
 
 
+# Tensor-pipe arithmetic of one B200 SM: a 128 x 128 x 16 bf16 tcgen05.mma retires in 64 cycles
+# (2 * 128 * 128 * 16 / 64 = 8,192 flop per clock per SM; a probe of back-to-back MMAs measured 67 cycles).
+SM_COUNT = 148
+BF16_FLOP_PER_CLK_PER_SM = 8192
+NOMINAL_BF16_TFLOPS = 2250.0      # datasheet dense bf16 figure
+
+
+def hw_tensor_peak_tflops(sm_mhz):
+    """Tensor-pipe ceiling at a given SM clock: SMs x flop/clk/SM x clock."""
+    return SM_COUNT * BF16_FLOP_PER_CLK_PER_SM * sm_mhz * 1e6 / 1e12
+
+
+def workload_config(workload, world=1, layers=0):
+    """The `config` object of the JSON line, the same in both arms."""
+    shape_name, prefix, suffix, pool_blocks = WORKLOADS[workload]
+    shape = synth.SHAPES[shape_name]
+    return {"workload": workload, "shape": shape.name, "layers": layers or shape.n_layers,
+            "prefix_tokens": prefix, "suffix_tokens": suffix, "block_size": shape.block_size, "pool_blocks": pool_blocks,
+            "block_ids": "seeded permutation (fragmented)", "parallelism": f"replicas x{world}",
+            "l2": "inputs larger than L2: each step streams every weight (>> 126 MB) between "
+                  "consecutive launches of any kernel; standalone pack/unpack rotate over disjoint block sets"}
+
+
 def peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -114,19 +137,38 @@ def oracle_copy_rates(shape, n_blocks):
     return 2.0 * wire.nbytes / (t1 - t0) / 1e9, 2.0 * wire.nbytes / (t2 - t1) / 1e9
 
 
-def cpu_baseline(shape, prefix, sample_tokens, repeats=1, suffix_blocks=0):
+def oracle_sample_tokens(prefix, cap, steps, warmup):
+    """Prefix tokens in the oracle's bounded sample: the whole prefix when the steps + warm-ups asked for fit in about
+    four minutes of host time (one layer over 4,096 tokens of the 32B shape takes about 17 s on 16 cores), else half
+    or a quarter of it.  Both arms size the sample with this function, so they time the same work."""
+    tokens = min(prefix, cap)
+    runs = steps + warmup
+    if runs > 13:
+        tokens = min(tokens, max(prefix // 2, 1))
+    if runs > 40:
+        tokens = min(tokens, max(prefix // 4, 1))
+    return tokens
+
+
+def oracle_sample_text(shape, prefix, sample_tokens):
+    part = "the whole prefix" if sample_tokens == prefix else f"the first {sample_tokens} of {prefix} prefix tokens"
+    return (f"one decoder layer (1 of {shape.n_layers}) of the fp64 numpy oracle over {part}; tokens/s extrapolated "
+            f"to {shape.n_layers} layers")
+
+
+def cpu_baseline(shape, prefix, sample_tokens, repeats=3, suffix_blocks=0):
+    """The oracle as it stands on the host cores: best of `repeats` runs of the bounded sample."""
     run = oracle_sample(shape, sample_tokens)
-    secs = min(run() for _ in range(repeats))
+    times = [run() for _ in range(repeats)]
+    secs = min(times)
     value = sample_tokens / (secs * shape.n_layers)
     extra = {}
     if suffix_blocks:
         pack, unpack = oracle_copy_rates(shape, suffix_blocks)
         extra = {"pack_gbs": pack, "unpack_gbs": unpack, "copy_sample": f"{suffix_blocks} suffix blocks, one thread"}
     return {**extra, "value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
-            "sample": f"one decoder layer (1 of {shape.n_layers}) of the fp64 numpy oracle over the first "
-                      f"{sample_tokens} of {prefix} prefix tokens, {secs:.2f} s; tokens/s extrapolated to "
-                      f"{shape.n_layers} layers",
-            "seconds": secs}
+            "sample": oracle_sample_text(shape, prefix, sample_tokens) + f"; best of {repeats} runs",
+            "seconds": secs, "seconds_all": [round(t, 3) for t in times]}
 
 
 def run_reference(args):
@@ -135,22 +177,22 @@ def run_reference(args):
         return 0
     shape_name, prefix, suffix, _ = WORKLOADS[args.workload]
     shape = synth.SHAPES[shape_name]
-    sample_tokens = min(prefix, args.ref_tokens)
+    warmup = max(args.ref_warmup, args.warmup if args.warmup_given else 0)
+    sample_tokens = oracle_sample_tokens(prefix, args.ref_tokens, args.steps, warmup)
     run = oracle_sample(shape, sample_tokens)
-    for _ in range(max(args.ref_warmup, args.warmup if args.warmup_given else 0)):
+    for _ in range(warmup):
         run()
     times = [run() for _ in range(args.steps)]
     secs = sum(times) / len(times)
     value = sample_tokens / (secs * shape.n_layers)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": max(args.ref_warmup, args.warmup if args.warmup_given else 0), "ms_per_step": secs * 1e3, "higher_is_better": True,
+        "steps": args.steps, "warmup": warmup, "ms_per_step": secs * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": args.workload, "prefix_tokens": prefix, "suffix_tokens": suffix,
-                   "step": f"one decoder layer of {shape.n_layers} over {sample_tokens} prefix tokens (bounded sample)"},
+        "config": workload_config(args.workload, world=args.gpus),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
-                         "sample": f"1 of {shape.n_layers} layers, {sample_tokens} of {prefix} prefix tokens, "
-                                   f"extrapolated to full depth"},
+                         "sample": oracle_sample_text(shape, prefix, sample_tokens) + f"; mean of {args.steps} steps",
+                         "best_value": sample_tokens / (min(times) * shape.n_layers)},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -281,17 +323,26 @@ def run_ours(args):
         merged = kv.kv_unpack_assemble(tgt, wire, logical, dst_ids, tgt_prefix, n, epoch=1, expected_epoch=1)
         kv.kv_decode_step(model, tgt, int(ids[n]), n, list(merged) + extra, logits, workspace=ws_d)
 
+    e2e_marks = []
+
     def step_e2e():
         # host buffers: token ids and tables are host arrays; the wire crosses the host (the link between
-        # source and target) and the logits are read back
+        # source and target) and the logits are read back.  Events split the step into its legs.
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+        ev[0].record(stream)
         kv.kv_prefill_prefix(model, tgt, ids[:prefix], tgt_prefix, workspace=ws_p)
         kv.kv_pack_blocks(src, src_suffix, wire)
+        ev[1].record(stream)
         wire_host.copy_(wire, non_blocking=True)
         wire2.copy_(wire_host, non_blocking=True)
+        ev[2].record(stream)
         merged = kv.kv_unpack_assemble(tgt, wire2, logical, dst_ids, tgt_prefix, n, epoch=1, expected_epoch=1)
         kv.kv_decode_step(model, tgt, int(ids[n]), n, list(merged) + extra, logits, workspace=ws_d)
+        ev[3].record(stream)
         logits_host.copy_(logits, non_blocking=True)
+        ev[4].record(stream)
         stream.synchronize()
+        e2e_marks.append(ev)
 
     def barrier():
         if world > 1:
@@ -373,7 +424,31 @@ def run_ours(args):
     kv.kv_check_device_status(ws_d)
 
     step_e2e()
+    e2e_marks.clear()
     e2e_ms = timed(step_e2e, args.steps)
+    legs = np.array([[a.elapsed_time(b) for a, b in zip(ev[:-1], ev[1:])] for ev in e2e_marks]).mean(axis=0)
+
+    # prefix-length sweep of the same shape (K/V-only prefill, 3 timed calls each after one warm-up call)
+    sweep = {}
+    if args.sweep and shape_name == "32b" and not args.layers:
+        for length in (512, 2048, 8192, 16384):
+            table = perm_tgt[: length // bs].copy()
+            ids_l = synth.token_ids(shape, seed + 7, length)
+            ws_l = model.workspace(kv.KV_OP_PREFILL, length)
+            kv.kv_prefill_prefix(model, tgt, ids_l, table, workspace=ws_l)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(3):
+                kv.kv_prefill_prefix(model, tgt, ids_l, table, workspace=ws_l)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            kv.kv_check_device_status(ws_l)
+            ms = e0.elapsed_time(e1) / 3
+            fl = prefill_flops(shape, length)
+            sweep[str(length)] = {"ms_per_prefix": round(ms, 3), "tokens_per_s": round(length / (ms * 1e-3), 1),
+                                  "tflops": round(fl / (ms * 1e-3) / 1e12, 1),
+                                  "bar_ms_60pct_of_burst": round(fl / (0.6 * peaks()["bf16_tflops"] * 1e12) * 1e3, 1)}
 
     if rank != 0:
         if world > 1:
@@ -391,40 +466,58 @@ def run_ours(args):
     gu_flops = 2.0 * prefix * shape.hidden * 2 * shape.ffn
     achieved = gu_flops / (gu_ms / max(gu_launches, 1) * 1e-3) / 1e12 if gu_ms > 0 else 0.0
     flops = prefill_flops(shape, prefix)
+    sm_mhz = clocks.get("sm_mhz") or 0.0
+    hw_peak = hw_tensor_peak_tflops(sm_mhz) if sm_mhz else None
+    traffic = NCU_TRAFFIC_BYTES.get(args.workload) if not args.layers else None
     roofline = {"bound": "tensor", "kernel": "gemm_tc_pair_kernel<SWIGLU, 256> (gate/up projection, cta_group::2)", "achieved": achieved,
                 "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": achieved / pk["bf16_tflops_sustained"],
-                "frac_of_burst_peak": achieved / pk["bf16_tflops"], "peak_source": pk["source"] + " (sustained)",
+                "peak_source": pk["source"] + " library bf16 matmul, sustained (the kernel is timed inside a long power-capped step)",
+                "frac_of_burst_peak": achieved / pk["bf16_tflops"],
+                "tensor_pipe_peak_at_sampled_clock": hw_peak,
+                "frac_of_tensor_pipe_at_sampled_clock": achieved / hw_peak if hw_peak else None,
+                "tensor_pipe_model": f"{SM_COUNT} SMs x {BF16_FLOP_PER_CLK_PER_SM} bf16 flop/clk/SM x median sampled SM clock",
+                "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS,
                 "flops_per_launch": gu_flops, "launches_timed": gu_launches,
-                "traffic": NCU_TRAFFIC_BYTES.get(args.workload) if not args.layers else None}
+                "traffic": traffic,
+                "traffic_source": ("ncu capture summarised in profiles/gemm_tc_pair_gate_up_32b-4k.md (same shape, one launch); "
+                                   "not measured in this run") if traffic else None}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": args.workload, "shape": shape.name, "layers": shape.n_layers,
-                   "prefix_tokens": prefix, "suffix_tokens": suffix, "block_size": bs, "pool_blocks": pool_blocks,
-                   "block_ids": "seeded permutation (fragmented)", "parallelism": f"replicas x{world}",
-                   "l2": "inputs larger than L2: each step streams every weight (>> 126 MB) between "
-                         "consecutive launches of any kernel; standalone pack/unpack rotate over disjoint block sets"},
+        "config": workload_config(args.workload, world=world, layers=args.layers),
         "clocks": clocks,
         "e2e": {"value": world * prefix / (e2e_ms / args.steps * 1e-3), "unit": UNIT,
                 "h2d_bytes_per_step": int(payload + 4 * (prefix + nb_prefix + nb_total + 1 + nb_suffix * 2)),
-                "d2h_bytes_per_step": int(payload + 4 * shape.vocab), "ms_per_step": e2e_ms / args.steps},
+                "d2h_bytes_per_step": int(payload + 4 * shape.vocab), "ms_per_step": e2e_ms / args.steps,
+                "prefill_pack_ms": float(legs[0]), "copy_ms": float(legs[1] + legs[3]),
+                "wire_d2h_h2d_ms": float(legs[1]), "logits_d2h_ms": float(legs[3]),
+                "unpack_decode_ms": float(legs[2]),
+                "note": "legs are CUDA-event times inside the end-to-end step (mean over the timed steps)"},
         "gpu_launches": int(launches),
         "roofline": roofline,
         "prefill": {"ms_per_prefix": prefill_ms, "tokens_per_s": prefix / (prefill_ms * 1e-3),
                     "tflops": flops / (prefill_ms * 1e-3) / 1e12,
                     "frac_of_bf16_burst_peak": flops / (prefill_ms * 1e-3) / 1e12 / pk["bf16_tflops"],
-                    "frac_of_bf16_sustained_peak": flops / (prefill_ms * 1e-3) / 1e12 / pk["bf16_tflops_sustained"]},
+                    "frac_of_bf16_sustained_peak": flops / (prefill_ms * 1e-3) / 1e12 / pk["bf16_tflops_sustained"],
+                    "frac_of_tensor_pipe_at_sampled_clock": flops / (prefill_ms * 1e-3) / 1e12 / hw_peak if hw_peak else None,
+                    "frac_of_nominal_2250": flops / (prefill_ms * 1e-3) / 1e12 / NOMINAL_BF16_TFLOPS},
         "pack": {"gbs": 2 * payload / (pack_ms * 1e-3) / 1e9, "frac_of_hbm": 2 * payload / (pack_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
                  "us": pack_ms * 1e3, "payload_bytes": payload,
-                 "timing": f"{pack_how} of {n_sets} launches over disjoint block sets"},
+                 "timing": f"{pack_how} of {n_sets} launches over disjoint block sets",
+                 "in_step_us": per_step["pack"][0] * 1e3,
+                 "frac_in_step": 2 * payload / (per_step["pack"][0] * 1e-3) / 1e9 / pk["hbm_gbs"]},
         "unpack": {"gbs": 2 * payload / (unpack_ms * 1e-3) / 1e9,
-                   "frac_of_hbm": 2 * payload / (unpack_ms * 1e-3) / 1e9 / pk["hbm_gbs"], "us": unpack_ms * 1e3},
+                   "frac_of_hbm": 2 * payload / (unpack_ms * 1e-3) / 1e9 / pk["hbm_gbs"], "us": unpack_ms * 1e3,
+                   "in_step_us": per_step["unpack"][0] * 1e3,
+                   "frac_in_step": 2 * payload / (per_step["unpack"][0] * 1e-3) / 1e9 / pk["hbm_gbs"]},
         "decode_step_ms": decode_ms,
         "decode_step_alone_ms": decode_alone_ms,
         "t0_analog_ms": per_step["unpack"][0] + decode_ms,
         "breakdown_ms_per_step": {k: round(v[0], 4) for k, v in per_step.items()},
     }
+    if sweep:
+        line["sweep"] = sweep
     # Algorithm 1 fed with the rates measured above (Section 4.2): prefill rate r_p, decode rate r_d of the
     # source (taken as this GPU's decode step), T_0 = assembly + first decode step, on two configured links.
     s_kv = kv.kv_bytes_per_token(shape.n_layers, shape.n_kv_heads, shape.head_dim, 2)
@@ -438,7 +531,9 @@ def run_ours(args):
         line["window"]["links"][name] = {"t_w_star": best["t_w"], "t_sit": best["t_sit"], "t_early": best["t_early"],
                                          "trigger_now": trig}
     if world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = cpu_baseline(synth.SHAPES[shape_name], prefix, min(prefix, args.ref_tokens),
+        ref_warmup = max(args.ref_warmup, args.warmup if args.warmup_given else 0)
+        line["cpu_baseline"] = cpu_baseline(synth.SHAPES[shape_name], prefix,
+                                            oracle_sample_tokens(prefix, args.ref_tokens, args.steps, ref_warmup),
                                             suffix_blocks=-(-suffix // synth.SHAPES[shape_name].block_size))
     print(json.dumps(line))
     if world > 1:
@@ -522,19 +617,29 @@ def run_stream_overlap(args):
 
 
 def run_batched_prefill(args):
-    """Concurrent migrations (Section 4.5): K prefixes rebuilt by one kv_prefill_prefix_batched call against K separate
-    kv_prefill_prefix calls, 32B shape."""
+    """Concurrent migrations (Section 4.5): 4 prefixes per GPU rebuilt by one kv_prefill_prefix_batched call against
+    separate kv_prefill_prefix calls, 32B shape.  With N GPUs the 4 N independent requests are dealt out over the ranks
+    (replicas.requests_of_rank), each rank rebuilds its share, no data-path collective."""
     import torch
+    import torch.distributed as dist
     import paper_2608_16477_b200 as kv
+    from paper_2608_16477_b200 import replicas
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     kv.load()
-    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
     shape = synth.SHAPES["32b"]
-    k_req, n = 4, 512
-    model, _ = build_model(kv, torch, shape)
+    n = 512
+    mine = replicas.requests_of_rank(4 * world, world, rank)
+    k_req = len(mine)
+    model, _ = build_model(kv, torch, shape, 1000 + rank)
     blocks_each = n // shape.block_size
     cache = kv.PagedCache(shape, k_req * blocks_each + 8, fill=0)
     perm = synth.block_permutation(3, k_req * blocks_each + 8)
-    ids = [synth.token_ids(shape, 10 + i, n) for i in range(k_req)]
+    ids = [synth.token_ids(shape, 10 + r, n) for r in mine]
     tabs = [perm[i * blocks_each:(i + 1) * blocks_each].copy() for i in range(k_req)]
 
     def separate():
@@ -547,22 +652,32 @@ def run_batched_prefill(args):
     def timed(fn):
         for _ in range(max(args.warmup, 3)):
             fn()
+        if world > 1:
+            dist.barrier()
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(args.steps):
             fn()
         e1.record()
+        if world > 1:
+            dist.barrier()
         torch.cuda.synchronize()
-        return e0.elapsed_time(e1) / args.steps
+        return replicas.max_over_ranks(e0.elapsed_time(e1) / args.steps, device="cuda")
     ms_sep, ms_bat = timed(separate), timed(batched)
-    line = {"metric": METRIC, "value": k_req * n / (ms_bat * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_bat, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": "batched-prefill", "shape": "32b", "requests": k_req, "prefix_tokens": n},
-            "batched_ms": ms_bat, "separate_calls_ms": ms_sep,
-            "separate_calls_tokens_per_s": k_req * n / (ms_sep * 1e-3), "gpu_launches": int(kv.kv_launch_count())}
-    print(json.dumps(line))
+    if rank == 0:
+        line = {"metric": METRIC, "value": replicas.whole_job_throughput(k_req * n, world, ms_bat), "unit": UNIT,
+                "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms_bat, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": "batched-prefill", "shape": "32b", "requests_per_gpu": k_req, "prefix_tokens": n,
+                           "parallelism": f"replicas x{world}: requests dealt out round-robin over the ranks"},
+                "batched_ms": ms_bat, "separate_calls_ms": ms_sep,
+                "separate_calls_tokens_per_s": replicas.whole_job_throughput(k_req * n, world, ms_sep),
+                "gpu_launches": int(kv.kv_launch_count())}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
     return 0
 
 
@@ -629,9 +744,11 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="32b-4k", choices=sorted(WORKLOADS) + ["pack-stress", "stream-overlap", "batched-prefill"])
     ap.add_argument("--layers", type=int, default=0, help="debug: reduced depth (invalid as a bench number)")
-    ap.add_argument("--ref-tokens", type=int, default=2048, help="prefix tokens in the oracle's bounded sample")
+    ap.add_argument("--ref-tokens", type=int, default=4096, help="prefix tokens in the oracle's bounded sample")
     ap.add_argument("--ref-warmup", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", dest="sweep", action="store_false",
+                    help="skip the prefix-length sweep (512 / 2,048 / 8,192 / 16,384 tokens) after the timed region")
     args = ap.parse_args()
     args.warmup_given = any(a == "--warmup" or a.startswith("--warmup=") for a in sys.argv[1:])
     if args.workload == "pack-stress" and args.impl != "reference":

@@ -122,8 +122,9 @@ int64_t kv_bytes_per_token(int32_t n_layers, int32_t n_kv_heads, int32_t head_di
  * prefill/decode call on it: KV_OK, or KV_ERR_DEVICE if a kernel's bounded wait ran out. */
 int32_t kv_check_device_status(const void *workspace_dev, void *stream);
 
-/* Synchronises `stream` and reports whether any pack/unpack kernel of this process gave up a bounded wait
- * (KV_ERR_DEVICE; the copy it belonged to is then incomplete).  KV_OK otherwise. */
+/* Synchronises `stream` and reports whether any pack/unpack kernel on the current device gave up a bounded wait
+ * since the last call of this function (KV_ERR_DEVICE; the copy it belonged to is then incomplete); the record is
+ * cleared by the call.  KV_OK otherwise. */
 int32_t kv_check_copy_status(void *stream);
 
 /* ---------------------------------------------------------------- the four operations */
@@ -186,7 +187,8 @@ int32_t kv_decode_step(kv_model *m, const kv_cache_desc *cache, int32_t token_id
 
 /* Batched forms over n_req requests (CSR offsets blk_offsets_host[0..n_req] into block_ids_host);
  * request r uses wire buffer wire_dev_ptrs_host[r].  Same semantics per request as above, without
- * the table assembly. */
+ * the table assembly.  All requests share ONE kernel launch (up to 7,680 blocks and 64 requests per launch;
+ * beyond that the list continues in further launches). */
 int32_t kv_pack_blocks_batched(const kv_cache_desc *src, int32_t n_req, const int32_t *blk_offsets_host,
                                const int32_t *block_ids_host, void *const *wire_dev_ptrs_host,
                                int32_t wire_layout, void *stream);
@@ -201,7 +203,8 @@ int32_t kv_unpack_blocks_batched(const kv_cache_desc *dst, int32_t n_req, const 
  * mode 0: out_dev bf16 [M, N] = A W^T.
  * mode 1: resid_dev fp32 [M, N] += A W^T (residual stream update).
  * mode 2: W is [2N, K] (gate | up); out_dev bf16 [M, N] = silu(A Wg^T) * (A Wu^T)  (SwiGLU).
- * K and N must be multiples of 8.  M is arbitrary.  mode | KV_GEMM_CTA_PAIR selects the kernel in which two CTAs
+ * K, lda and N must be multiples of 8, lda >= K; out_dev and resid_dev 16-byte aligned.  M is arbitrary.
+ * mode | KV_GEMM_CTA_PAIR selects the kernel in which two CTAs
  * (two SMs) share one 256 x 256 tile through tcgen05 cta_group::2; results are identical. */
 #define KV_GEMM_CTA_PAIR 0x100
 int32_t kv_op_gemm(const void *a_dev, int32_t lda, const void *w_dev, int32_t m, int32_t n, int32_t k,
@@ -214,19 +217,24 @@ int32_t kv_op_gemm(const void *a_dev, int32_t lda, const void *w_dev, int32_t m,
 int32_t kv_op_gemv(const void *w_dev, const float *x_dev, int32_t n, int32_t k, int32_t mode, const void *gain_dev,
                    float eps, float *y_dev, void *stream);
 
-/* Diagnostics.  The same projection computed by a plain CUDA-core kernel (no tensor cores, no TMA):
- * an independent on-device cross-check of kv_op_gemm for unit tests.  No operation above uses it. */
-int32_t kv_op_gemm_reference(const void *a_dev, int32_t lda, const void *w_dev, int32_t m, int32_t n, int32_t k,
-                             int32_t mode, void *out_dev, float *resid_dev, void *stream);
+/* Which kernel and tile the projection launcher uses for an m-row problem with n output columns: *cta_pair_out = 1
+ * when two CTAs share a 256-row tile (tcgen05 cta_group::2), 0 for the one-CTA kernel; *tile_width_out = columns of W
+ * per tile (128..256; a SwiGLU tile holds tile_width/2 gate and tile_width/2 up rows).  mode 0..2 as in kv_op_gemm,
+ * 3 = the fused QKV projection (head_dim required: tiles hold whole heads).  Read-only; depends on the current
+ * device's SM count.  Lets a test or a report state which instantiation a given problem size runs. */
+int32_t kv_gemm_plan(int32_t m, int32_t n, int32_t mode, int32_t head_dim, int32_t *cta_pair_out,
+                     int32_t *tile_width_out);
 
 /* RMSNorm of fp32 rows x [rows, dim] with bf16 gain -> bf16 out [rows, dim]. */
 int32_t kv_op_rmsnorm(const float *x_dev, const void *gain_dev, int32_t rows, int32_t dim, float eps,
                       void *out_dev, void *stream);
 
-/* Causal GQA flash attention of a prefill chunk.  qkv_dev bf16 [T, (Hq+2Hkv) d] holds post-RoPE Q and
- * K and V of positions pos0..pos0+T-1; earlier positions [0,pos0) are read from the paged cache through
- * block_table_dev.  out_dev bf16 [T, Hq d]. */
-int32_t kv_op_attention_prefill(const void *qkv_dev, int32_t n_tokens, int32_t pos0,
+/* Causal GQA flash attention of a prefill chunk (step 4 of a decoder layer inside kv_prefill_prefix; Section 4.5 for
+ * pos0 > 0).  qkv_ctx_dev bf16 [pos0 + T, (Hq+2Hkv) d], one row per context position: rows [pos0, pos0+T) hold the
+ * chunk's post-RoPE Q and K and its V.  With pos0 > 0 (a multiple of block_size) the call first copies the K and V of
+ * positions [0,pos0) from the paged cache (through block_table_dev) into the K and V columns of rows [0,pos0); the Q
+ * columns of those rows are not touched or read.  out_dev bf16 [T, Hq d].  head_dim 64 or 128. */
+int32_t kv_op_attention_prefill(void *qkv_ctx_dev, int32_t n_tokens, int32_t pos0,
                                 int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
                                 const kv_cache_desc *cache, int32_t layer, const int32_t *block_table_dev,
                                 void *out_dev, int32_t *status_dev, void *stream);

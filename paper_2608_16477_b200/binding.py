@@ -17,7 +17,7 @@ EXPORTS = [
     "kv_model_create", "kv_model_destroy", "kv_workspace_bytes", "kv_status_string", "kv_last_cuda_error",
     "kv_bytes_per_token", "kv_check_device_status", "kv_prefill_prefix", "kv_pack_blocks",
     "kv_unpack_assemble", "kv_decode_step", "kv_pack_blocks_batched", "kv_unpack_blocks_batched",
-    "kv_op_gemm", "kv_op_gemm_reference", "kv_op_rmsnorm",
+    "kv_op_gemm", "kv_gemm_plan", "kv_op_rmsnorm",
     "kv_op_attention_prefill", "kv_paged_attention_scratch_bytes", "kv_op_paged_attention", "kv_fill_pattern",
     "kv_profile_enable", "kv_profile_read", "kv_launch_count", "kv_op_paged_attention_noalloc", "kv_check_copy_status", "kv_op_gemv",
     "kv_window_evaluate", "kv_window_select", "kv_window_waste_bound", "kv_ewma", "kv_prefill_prefix_batched",
@@ -101,7 +101,7 @@ def load(build_if_missing: bool = True):
         "kv_pack_blocks_batched": (i32, [C.POINTER(CacheDesc), i32, pi32, pi32, C.POINTER(vp), i32, vp]),
         "kv_unpack_blocks_batched": (i32, [C.POINTER(CacheDesc), i32, pi32, pi32, C.POINTER(vp), i32, vp]),
         "kv_op_gemm": (i32, [vp, i32, vp, i32, i32, i32, i32, vp, vp, vp, vp]),
-        "kv_op_gemm_reference": (i32, [vp, i32, vp, i32, i32, i32, i32, vp, vp, vp]),
+        "kv_gemm_plan": (i32, [i32, i32, i32, i32, pi32, pi32]),
         "kv_op_rmsnorm": (i32, [vp, vp, i32, i32, C.c_float, vp, vp]),
         "kv_op_attention_prefill": (i32, [vp, i32, i32, i32, i32, i32, C.POINTER(CacheDesc), i32, vp, vp, vp, vp]),
         "kv_paged_attention_scratch_bytes": (i64, [i32, i32, i32]),
@@ -231,11 +231,11 @@ class Model:
         import torch
         need = kv_workspace_bytes(self, op, max_tokens)
         cur = self._ws.get(op)
-        if cur is None or cur.numel() < need:
+        if cur is None or cur.numel() - ((-cur.data_ptr()) % 1024) < need:
             cur = torch.empty(need + 1024, dtype=torch.uint8, device=self.device)
             self._ws[op] = cur
-        off = (-cur.data_ptr()) % 1024
-        return cur[off:off + need] if need <= cur.numel() - off else cur
+        off = (-cur.data_ptr()) % 1024            # the library wants a 1 KiB-aligned base
+        return cur[off:off + need]
 
     def __del__(self):
         try:
@@ -336,11 +336,11 @@ def kv_op_gemm(a, w, mode: int, out=None, resid=None, status=None, stream=None, 
                              _stream(stream)), "kv_op_gemm")
 
 
-def kv_op_gemm_reference(a, w, mode: int, out=None, resid=None, stream=None, n=None):
-    m, k = a.shape
-    n = n if n is not None else (w.shape[0] // 2 if mode == 2 else w.shape[0])
-    _check(load().kv_op_gemm_reference(_ptr(a), a.stride(0), _ptr(w), m, n, k, mode, _ptr(out), _ptr(resid),
-                                       _stream(stream)), "kv_op_gemm_reference")
+def kv_gemm_plan(m: int, n: int, mode: int, head_dim: int = 0):
+    """(cta_pair, tile_width) the projection launcher picks for an m x n problem (mode 3 = fused QKV)."""
+    pair, bn = C.c_int32(), C.c_int32()
+    _check(load().kv_gemm_plan(m, n, mode, head_dim, C.byref(pair), C.byref(bn)), "kv_gemm_plan")
+    return bool(pair.value), int(bn.value)
 
 
 def kv_op_rmsnorm(x, gain, eps: float, out, stream=None):
@@ -348,9 +348,11 @@ def kv_op_rmsnorm(x, gain, eps: float, out, stream=None):
            "kv_op_rmsnorm")
 
 
-def kv_op_attention_prefill(qkv, n_q_heads, n_kv_heads, head_dim, out, pos0=0, cache=None, layer=0,
+def kv_op_attention_prefill(qkv_ctx, n_q_heads, n_kv_heads, head_dim, out, pos0=0, cache=None, layer=0,
                             block_table_dev=None, status=None, stream=None):
-    _check(load().kv_op_attention_prefill(_ptr(qkv), qkv.shape[0], pos0, n_q_heads, n_kv_heads, head_dim,
+    """qkv_ctx has pos0 + T rows (the chunk's rows last); with pos0 > 0 the call fills the K/V columns of the first
+    pos0 rows from the cache."""
+    _check(load().kv_op_attention_prefill(_ptr(qkv_ctx), qkv_ctx.shape[0] - pos0, pos0, n_q_heads, n_kv_heads, head_dim,
                                           C.byref(cache.desc) if cache is not None else None, layer,
                                           _ptr(block_table_dev), _ptr(out), _ptr(status), _stream(stream)),
            "kv_op_attention_prefill")

@@ -10,10 +10,10 @@ CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libkvrebuild.so")
 STAMP = os.path.join(PKG_DIR, "build", "stamp.txt")
 
-SOURCES = ["api.cu", "copy_pages.cu", "elementwise.cu", "decode.cu", "gemm_simt.cu", "gemm_tcgen05.cu", "gemm_tcgen05_pair.cu",
-           "attention_prefill.cu", "attention_tcgen05.cu", "paged_attention_noalloc.cu", "window.cu"]
+SOURCES = ["api.cu", "copy_pages.cu", "elementwise.cu", "decode.cu", "gemm_tcgen05.cu", "gemm_tcgen05_pair.cu",
+           "attention_tcgen05.cu", "paged_attention_noalloc.cu", "window.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "--use_fast_math", "-Xcompiler", "-fPIC", "-Xptxas", "-v"] + os.environ.get("KV_NVCC_EXTRA", "").split()
+              "--use_fast_math", "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 
 
 def _nvcc() -> str:

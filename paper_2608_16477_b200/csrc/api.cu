@@ -202,18 +202,7 @@ DecodeWs carve_decode(const kv_model_desc &d, void *base, int max_ctx, int block
   return w;
 }
 
-int check_cache(const kv_cache_desc *c) {
-  if (c == nullptr || c->base_dev == nullptr) return KV_ERR_ARG;
-  if (c->num_blocks <= 0 || c->block_size <= 0 || c->n_layers <= 0 || c->n_kv_heads <= 0 || c->head_dim <= 0)
-    return KV_ERR_ARG;
-  if (c->elem_bytes != 2) return KV_ERR_SHAPE;
-  const long long page = (long long)c->block_size * c->n_kv_heads * c->head_dim * 2;
-  if (page % 16 != 0) return KV_ERR_SHAPE;
-  if (((uintptr_t)c->base_dev & 15) || (c->layer_stride & 15) || (c->kv_stride & 15) || (c->block_stride & 15))
-    return KV_ERR_ARG;
-  if (c->block_stride < page || c->kv_stride <= 0 || c->layer_stride <= 0) return KV_ERR_ARG;
-  return KV_OK;
-}
+int check_cache(const kv_cache_desc *c) { return check_cache_desc(c); }
 
 int check_cache_vs_model(const kv_cache_desc *c, const kv_model_desc &d) {
   int rc = check_cache(c);
@@ -237,21 +226,13 @@ long long wire_bytes_needed(const kv_cache_desc *c, int n_blocks) {
   return (long long)n_blocks * c->n_layers * 2 * c->block_size * c->n_kv_heads * c->head_dim * 2;
 }
 
-// Which projections run on the CTA-pair kernel (bit mask over GemmMode), settable for experiments through
-// the KV_GEMM_PAIR_MODES environment variable.  Up to 128 rows (one row tile) the one-CTA kernel is used; from
-// there on the pair kernel was as fast or faster for every projection measured (512 to 16,384 rows).
-int pair_mode_mask() {
-  static int mask = -1;
-  if (mask < 0) {
-    const char *e = getenv("KV_GEMM_PAIR_MODES");
-    mask = e ? atoi(e) : 15;    // every mode
-  }
-  return mask;
-}
+// Up to 128 rows (one row tile) the one-CTA kernel runs; from there on the CTA-pair kernel was as fast or faster
+// for every projection measured (512 to 16,384 rows).
+inline bool gemm_uses_pair(int rows) { return rows > 128; }
 
 int run_gemm(const kv_model *, const bf16 *a, int lda, const bf16 *w, int rows, int n, int k, int mode, bf16 *out,
              float *resid, DeviceStatus *status, cudaStream_t st, const QkvRopeArgs *qa = nullptr) {
-  if (rows > 128 && ((pair_mode_mask() >> mode) & 1))
+  if (gemm_uses_pair(rows))
     return gemm_tc_pair(a, lda, w, rows, n, k, mode, out, resid, reinterpret_cast<int *>(status), st, qa);
   return gemm_tc(a, lda, w, rows, n, k, mode, out, resid, reinterpret_cast<int *>(status), st, qa);
 }
@@ -375,7 +356,6 @@ int prefill_layers(kv_model *m, const CacheView &cv, PrefillWs &w, int total_row
   const int q_dim = d.n_q_heads * d.head_dim;
   { ProfScope ps(PROF_ROPE_STORE, st); KV_TRY(rope_table(w.rope, pos0, t, d.head_dim, d.rope_base, st, row_pos)); }
   // the qkv buffer has one row per context position; the chunk's rows start at pos0
-  const bool tc_attention = attention_tc_supported(d.n_q_heads, d.n_kv_heads, d.head_dim);
   bf16 *qkv_chunk = w.qkv + (long long)pos0 * qkv_dim;
   { ProfScope ps(PROF_EMBED, st); KV_TRY(embed_rows(m->embed, w.ids, t, d.hidden, w.x, st)); }
   for (int l = 0; l < d.n_layers; ++l) {
@@ -402,14 +382,9 @@ int prefill_layers(kv_model *m, const CacheView &cv, PrefillWs &w, int total_row
       for (const PrefillSegment &sg : segs) {
         bf16 *seg_qkv = w.qkv + (long long)sg.row0 * qkv_dim;     // rows of this request (its context starts here)
         bf16 *seg_out = w.attn + (long long)sg.row0 * q_dim;
-        if (tc_attention) {
-          KV_TRY(gather_prefix_kv(seg_qkv, pos0, d.n_q_heads, d.n_kv_heads, d.head_dim, cv, l, w.table, st));
-          KV_TRY(attention_prefill_tc(seg_qkv, sg.n_tokens, pos0, d.n_q_heads, d.n_kv_heads, d.head_dim, seg_out,
-                                      reinterpret_cast<int *>(w.status), st));
-        } else {
-          KV_TRY(attention_prefill(seg_qkv + (long long)pos0 * qkv_dim, sg.n_tokens, pos0, d.n_q_heads, d.n_kv_heads,
-                                   d.head_dim, cv, l, w.table, seg_out, reinterpret_cast<int *>(w.status), st));
-        }
+        KV_TRY(gather_prefix_kv(seg_qkv, pos0, d.n_q_heads, d.n_kv_heads, d.head_dim, cv, l, w.table, st));
+        KV_TRY(attention_prefill_tc(seg_qkv, sg.n_tokens, pos0, d.n_q_heads, d.n_kv_heads, d.head_dim, seg_out,
+                                    reinterpret_cast<int *>(w.status), st));
       }
     }
     { ProfScope ps(PROF_GEMM_O, st); KV_TRY(run_gemm(m, w.attn, q_dim, m->w_o[l], t, d.hidden, q_dim, GEMM_RESID_F32, nullptr, w.x, w.status, st)); }
@@ -550,8 +525,8 @@ int32_t kv_pack_blocks(const kv_cache_desc *src, const int32_t *block_ids_host, 
   if (wire_bytes < wire_bytes_needed(src, n_blocks)) return KV_ERR_WIRE_SIZE;
   if (n_blocks == 0) return KV_OK;
   ProfScope ps(PROF_PACK, (cudaStream_t)stream);
-  return copy_pages(make_view(src), src->n_layers, block_ids_host, n_blocks, (char *)wire_dev, wire_layout, n_blocks,
-                    0, true, (cudaStream_t)stream);
+  const CopyRequest req{block_ids_host, n_blocks, (char *)wire_dev};
+  return copy_pages(make_view(src), src->n_layers, &req, 1, wire_layout, true, (cudaStream_t)stream);
 }
 
 int32_t kv_unpack_assemble(const kv_cache_desc *dst, const void *wire_dev, int64_t wire_bytes, int32_t wire_layout,
@@ -586,8 +561,8 @@ int32_t kv_unpack_assemble(const kv_cache_desc *dst, const void *wire_dev, int64
   if (wire_bytes < wire_bytes_needed(dst, n_suffix)) return KV_ERR_WIRE_SIZE;
   if (n_suffix > 0) {
     ProfScope ps(PROF_UNPACK, (cudaStream_t)stream);
-    rc = copy_pages(make_view(dst), dst->n_layers, dst_ids, n_suffix, (char *)const_cast<void *>(wire_dev), wire_layout,
-                    n_suffix, 0, false, (cudaStream_t)stream);
+    const CopyRequest req{dst_ids, n_suffix, (char *)const_cast<void *>(wire_dev)};
+    rc = copy_pages(make_view(dst), dst->n_layers, &req, 1, wire_layout, false, (cudaStream_t)stream);
     if (rc != KV_OK) return rc;
   }
   for (int i = 0; i < n_prefix; ++i) merged_out[i] = prefix_table[i];
@@ -610,15 +585,12 @@ static int32_t batched(const kv_cache_desc *c, int32_t n_req, const int32_t *off
   // destinations must not alias across the whole batch; sources may repeat
   rc = check_ids(ids, offs[n_req], c->num_blocks, !to_wire);
   if (rc != KV_OK) return rc;
-  for (int r = 0; r < n_req; ++r) {
-    const int nb = offs[r + 1] - offs[r];
-    if (nb == 0) continue;
-    ProfScope ps(to_wire ? PROF_PACK : PROF_UNPACK, (cudaStream_t)stream);
-    rc = copy_pages(make_view(c), c->n_layers, ids + offs[r], nb, (char *)wires[r], layout, nb, 0, to_wire,
-                    (cudaStream_t)stream);
-    if (rc != KV_OK) return rc;
-  }
-  return KV_OK;
+  std::vector<CopyRequest> reqs;
+  for (int r = 0; r < n_req; ++r)
+    if (offs[r + 1] > offs[r]) reqs.push_back({ids + offs[r], offs[r + 1] - offs[r], (char *)wires[r]});
+  if (reqs.empty()) return KV_OK;
+  ProfScope ps(to_wire ? PROF_PACK : PROF_UNPACK, (cudaStream_t)stream);
+  return copy_pages(make_view(c), c->n_layers, reqs.data(), (int)reqs.size(), layout, to_wire, (cudaStream_t)stream);
 }
 
 int32_t kv_pack_blocks_batched(const kv_cache_desc *src, int32_t n_req, const int32_t *blk_offsets_host,
@@ -639,7 +611,10 @@ int32_t kv_op_gemm(const void *a_dev, int32_t lda, const void *w_dev, int32_t m,
   const bool pair = (mode & KV_GEMM_CTA_PAIR) != 0;
   mode &= ~KV_GEMM_CTA_PAIR;
   if (a_dev == nullptr || w_dev == nullptr || mode < 0 || mode > 2) return KV_ERR_ARG;
+  if (m < 0 || n <= 0 || k <= 0 || lda < k) return KV_ERR_ARG;
   if ((mode == GEMM_RESID_F32 && resid_dev == nullptr) || (mode != GEMM_RESID_F32 && out_dev == nullptr)) return KV_ERR_ARG;
+  // the epilogues store 16-byte vectors (bf16 output) and update the residual stream as float4
+  if (((uintptr_t)out_dev & 15) || ((uintptr_t)resid_dev & 15) || ((uintptr_t)status_dev & 3)) return KV_ERR_ARG;
   if (pair)
     return gemm_tc_pair((const bf16 *)a_dev, lda, (const bf16 *)w_dev, m, n, k, mode, (bf16 *)out_dev, resid_dev,
                         status_dev, (cudaStream_t)stream);
@@ -647,11 +622,16 @@ int32_t kv_op_gemm(const void *a_dev, int32_t lda, const void *w_dev, int32_t m,
                  (cudaStream_t)stream);
 }
 
-int32_t kv_op_gemm_reference(const void *a_dev, int32_t lda, const void *w_dev, int32_t m, int32_t n, int32_t k,
-                             int32_t mode, void *out_dev, float *resid_dev, void *stream) {
-  if (a_dev == nullptr || w_dev == nullptr || mode < 0 || mode > 2) return KV_ERR_ARG;
-  return gemm_simt((const bf16 *)a_dev, lda, (const bf16 *)w_dev, m, n, k, mode, (bf16 *)out_dev, resid_dev,
-                   (cudaStream_t)stream);
+int32_t kv_gemm_plan(int32_t m, int32_t n, int32_t mode, int32_t head_dim, int32_t *cta_pair_out,
+                     int32_t *tile_width_out) {
+  if (m <= 0 || n <= 0 || mode < 0 || mode > GEMM_QKV_ROPE || cta_pair_out == nullptr || tile_width_out == nullptr)
+    return KV_ERR_ARG;
+  if (mode == GEMM_QKV_ROPE && head_dim != 64 && head_dim != 128) return KV_ERR_SHAPE;
+  const int sms = sm_count(current_device());
+  const int hd = mode == GEMM_QKV_ROPE ? head_dim : 0;
+  *cta_pair_out = gemm_uses_pair(m) ? 1 : 0;
+  *tile_width_out = gemm_uses_pair(m) ? gemm_tc_pair_tile_width(m, n, sms, mode, hd) : gemm_tc_tile_width(m, n, sms, mode, hd);
+  return KV_OK;
 }
 
 int32_t kv_op_gemv(const void *w_dev, const float *x_dev, int32_t n, int32_t k, int32_t mode, const void *gain_dev,
@@ -671,21 +651,24 @@ int32_t kv_op_rmsnorm(const float *x_dev, const void *gain_dev, int32_t rows, in
   return rmsnorm_rows(x_dev, (const bf16 *)gain_dev, rows, dim, eps, (bf16 *)out_dev, (cudaStream_t)stream);
 }
 
-int32_t kv_op_attention_prefill(const void *qkv_dev, int32_t n_tokens, int32_t pos0, int32_t n_q_heads,
+int32_t kv_op_attention_prefill(void *qkv_ctx_dev, int32_t n_tokens, int32_t pos0, int32_t n_q_heads,
                                 int32_t n_kv_heads, int32_t head_dim, const kv_cache_desc *cache, int32_t layer,
                                 const int32_t *block_table_dev, void *out_dev, int32_t *status_dev, void *stream) {
-  if (qkv_dev == nullptr || out_dev == nullptr || n_tokens < 0 || pos0 < 0) return KV_ERR_ARG;
-  CacheView cv;
-  memset(&cv, 0, sizeof(cv));
+  if (qkv_ctx_dev == nullptr || out_dev == nullptr || n_tokens < 0 || pos0 < 0 || n_q_heads <= 0 || n_kv_heads <= 0)
+    return KV_ERR_ARG;
+  if (((uintptr_t)qkv_ctx_dev & 15) || ((uintptr_t)out_dev & 15)) return KV_ERR_ARG;
+  if ((head_dim != 64 && head_dim != 128) || n_q_heads % n_kv_heads != 0) return KV_ERR_SHAPE;
   if (pos0 > 0) {
     int rc = check_cache(cache);
     if (rc != KV_OK) return rc;
     if (block_table_dev == nullptr || layer < 0 || layer >= cache->n_layers) return KV_ERR_ARG;
     if (cache->n_kv_heads != n_kv_heads || cache->head_dim != head_dim) return KV_ERR_SHAPE;
-    cv = make_view(cache);
+    if (pos0 % cache->block_size != 0) return KV_ERR_SPLIT_UNALIGNED;
+    KV_TRY(gather_prefix_kv((bf16 *)qkv_ctx_dev, pos0, n_q_heads, n_kv_heads, head_dim, make_view(cache), layer,
+                            block_table_dev, (cudaStream_t)stream));
   }
-  return attention_prefill((const bf16 *)qkv_dev, n_tokens, pos0, n_q_heads, n_kv_heads, head_dim, cv, layer,
-                           block_table_dev, (bf16 *)out_dev, status_dev, (cudaStream_t)stream);
+  return attention_prefill_tc((const bf16 *)qkv_ctx_dev, n_tokens, pos0, n_q_heads, n_kv_heads, head_dim,
+                              (bf16 *)out_dev, status_dev, (cudaStream_t)stream);
 }
 
 int64_t kv_paged_attention_scratch_bytes(int32_t n_q_heads, int32_t head_dim, int32_t n_ctx) {
@@ -699,6 +682,8 @@ int32_t kv_op_paged_attention(const float *q_dev, int32_t n_q_heads, const kv_ca
   if (q_dev == nullptr || block_table_dev == nullptr || scratch_dev == nullptr || out_dev == nullptr || n_ctx <= 0 ||
       n_q_heads <= 0)
     return KV_ERR_ARG;
+  // the kernels read q as float2 and write fp32 partials and outputs
+  if (((uintptr_t)q_dev & 7) || ((uintptr_t)out_dev & 3) || ((uintptr_t)scratch_dev & 15)) return KV_ERR_ARG;
   int rc = check_cache(cache);
   if (rc != KV_OK) return rc;
   if (layer < 0 || layer >= cache->n_layers || n_q_heads % cache->n_kv_heads != 0 ||

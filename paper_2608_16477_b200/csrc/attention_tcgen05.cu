@@ -3,7 +3,8 @@
 // prefix (gathered from its pages), rows [pos0, pos0 + T) the chunk's post-RoPE Q, K and V.
 //
 // A work item is ONE 128-row query tile of TWO query heads that share a KV head (tiles "a" and "b"), so
-// every K/V tile fetched by TMA feeds both.
+// every K/V tile fetched by TMA feeds both.  A KV head with an odd number of query heads pairs its last
+// query head with itself: both tiles then compute and store the same rows.
 //
 //   warp 0      TMA producer of Q (once per item) and of the K and V tiles (128 keys each).
 //   warps 1, 2  S = Q K^T of tile a and of tile b (both operands K-major in shared memory); warp 1 also
@@ -41,14 +42,6 @@ constexpr float kRescaleThreshold = 8.0f;
 // first launch and refuses to launch otherwise (compiled = 168 here: 256 x 48 = 128 x 96).
 constexpr int kRegsOther = 72;      // registers per thread of warps 0-3 after the hand-back
 constexpr int kRegsSoftmax = 216;   // registers per thread of the softmax warps
-
-#ifdef KV_ATTN_TRACE
-__device__ long long g_attn_trace[64 * 32];
-#define KV_ATRACE(slot, idx) \
-  do { if (blockIdx.x == 0 && (idx) < 64) g_attn_trace[(idx) * 32 + (slot)] = clock64(); } while (0)
-#else
-#define KV_ATRACE(slot, idx) do { } while (0)
-#endif
 
 enum AttnTag { ATAG_Q = 11, ATAG_K_EMPTY = 12, ATAG_K = 13, ATAG_V = 14, ATAG_S = 15, ATAG_P = 16, ATAG_O = 17,
                ATAG_V_EMPTY = 18, ATAG_S_FREE = 19, ATAG_PV = 20, ATAG_QK_ISSUED = 21 };
@@ -91,6 +84,74 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   return *reinterpret_cast<uint32_t *>(&h);
 }
 
+// ---- packed fp32 pairs (two floats in one 64-bit register pair, one instruction for both) and 3-input max:
+// they halve the instruction count of the softmax's scaling, row sums and running maximum.
+__device__ __forceinline__ uint64_t pk2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpk2(uint64_t v, float &lo, float &hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2_rm(uint64_t a, uint64_t b) {      // rounds towards minus infinity
+  uint64_t d;
+  asm("add.rm.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// 2^x for a pair on the FMA and integer pipes instead of the special-function unit: x = n + f with n = floor(x)
+// (taken from the mantissa of x + 1.5 * 2^23 added with rounding towards minus infinity) and f in [0, 1),
+// 2^f by a cubic (coefficients fitted for minimal relative error with p(0) = 1 and p(1) = 2: 1.0e-4, twenty times
+// below the bf16 rounding the probabilities get anyway), then n is added into the exponent field.  Arguments are
+// clamped at -126, so masked scores (minus infinity) come out as 2^-126 instead of 0: eight orders of magnitude
+// below anything a bf16 sum or product can notice.
+#ifndef KV_ATTN_POLY_PAIRS
+#define KV_ATTN_POLY_PAIRS 4     // pairs per 16-pair chunk whose exponentials take this path (4: a quarter of all)
+#endif
+constexpr int kPolyPairs = KV_ATTN_POLY_PAIRS;
+__device__ __forceinline__ void exp2_pair_fma(uint64_t x2, float &p0, float &p1) {
+  float x0, x1;
+  unpk2(x2, x0, x1);
+  const uint64_t xc = pk2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
+  const uint64_t magic = pk2(12582912.f, 12582912.f);
+  const uint64_t t = add2_rm(xc, magic);
+  const uint64_t f = sub2(xc, sub2(t, magic));
+  uint64_t p = fma2(f, pk2(0.07826797f, 0.07826797f), pk2(0.22630768f, 0.22630768f));
+  p = fma2(p, f, pk2(0.69542435f, 0.69542435f));
+  p = fma2(p, f, pk2(1.f, 1.f));
+  float q0, q1, t0, t1;
+  unpk2(p, q0, q1);
+  unpk2(t, t0, t1);
+  p0 = __int_as_float(__float_as_int(q0) + (__float_as_int(t0) << 23));
+  p1 = __int_as_float(__float_as_int(q1) + (__float_as_int(t1) << 23));
+}
+
 // Shared memory: two Q tiles, a ring of K tiles and a ring of V tiles.
 template <int D>
 struct AttnSmem {
@@ -127,7 +188,8 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int group = n_q_heads / n_kv_heads;
-  const int pairs = n_q_heads / 2;
+  const int pairs_per_group = (group + 1) / 2;
+  const int pairs = n_kv_heads * pairs_per_group;
   const int m_tiles = (n_tokens + kBM - 1) / kBM;
   const int n_items = m_tiles * pairs;
   const int n_ctx = pos0 + n_tokens;
@@ -141,19 +203,20 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
     return base + ((k & 1) ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)blockIdx.x);
   };
   struct Item {
-    int m0, n_kv, head_a, q_col0, q_col1, k_col, v_col;
+    int m0, n_kv, head_a, head_b, q_col0, q_col1, k_col, v_col;
   };
   auto get_item = [&](int it) {
     Item w;
     const int m_tile = m_tiles - 1 - it / pairs;
     const int pair = it % pairs;
-    w.head_a = 2 * pair;
-    const int kv_head = w.head_a / group;
+    const int kv_head = pair / pairs_per_group;
+    w.head_a = kv_head * group + 2 * (pair % pairs_per_group);
+    w.head_b = min(w.head_a + 1, kv_head * group + group - 1);
     w.m0 = m_tile * kBM;                                    // first chunk row of this tile
     // causal: key tiles up to the one holding the last row's own position
     w.n_kv = min((n_ctx + kBN - 1) / kBN, (pos0 + w.m0 + kBM - 1) / kBN + 1);
     w.q_col0 = w.head_a * D;
-    w.q_col1 = w.q_col0 + D;
+    w.q_col1 = w.head_b * D;
     w.k_col = (n_q_heads + kv_head) * D;
     w.v_col = (n_q_heads + n_kv_heads + kv_head) * D;
     return w;
@@ -335,7 +398,6 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
         ok = tc::mbar_wait(bar(B_S, t), s & 1, abort_flag, status, ATAG_S);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
-        if (quarter == 0 && lane == 0) KV_ATRACE(t * 4 + 0, s);
         tc::tc_fence_after();
         const bool diag = (j * kBN + kBN - 1 > pos0 + m0);   // tile reaches past the first row's position
         const int limit = qi - j * kBN;              // keys with column > limit are masked
@@ -349,22 +411,26 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
         tc::tc_fence_before();
         tc::mbar_arrive(bar(B_S_FREE, t));
         float mx = -INFINITY;
-        if (!diag) {
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            mx = fmaxf(mx, fmaxf(fmaxf(__uint_as_float(r0[i]), __uint_as_float(r1[i])),
-                                 fmaxf(__uint_as_float(r2[i]), __uint_as_float(r3[i]))));
-          }
-        } else {
+        if (diag) {
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
             if (i > limit) r0[i] = 0xff800000u;        // -inf
             if (32 + i > limit) r1[i] = 0xff800000u;
             if (64 + i > limit) r2[i] = 0xff800000u;
             if (96 + i > limit) r3[i] = 0xff800000u;
-            mx = fmaxf(mx, fmaxf(fmaxf(__uint_as_float(r0[i]), __uint_as_float(r1[i])),
-                                 fmaxf(__uint_as_float(r2[i]), __uint_as_float(r3[i]))));
           }
+        }
+        {
+          // four independent chains of 3-input maxima (16 dependent steps each instead of 64 in a row)
+          float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+          for (int i = 0; i < 32; i += 2) {
+            m0 = max3(m0, __uint_as_float(r0[i]), __uint_as_float(r0[i + 1]));
+            m1 = max3(m1, __uint_as_float(r1[i]), __uint_as_float(r1[i + 1]));
+            m2 = max3(m2, __uint_as_float(r2[i]), __uint_as_float(r2[i + 1]));
+            m3 = max3(m3, __uint_as_float(r3[i]), __uint_as_float(r3[i + 1]));
+          }
+          mx = fmaxf(max3(m0, m1, m2), m3);
         }
         mx *= scale_log2;
         bool rescale = false;
@@ -379,15 +445,22 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
         }
         // probabilities as packed bf16 (two keys per 32-bit column); masked scores are -inf -> 0.  The whole row is
         // exponentiated before the wait for the P columns, so that the wait finds P V_{j-1} done.
-        const float neg_m = -m_ref;
-        float sum0 = 0.f, sum1 = 0.f;
+        const uint64_t scale2 = pk2(scale_log2, scale_log2), neg_m2 = pk2(-m_ref, -m_ref);
+        uint64_t sum2 = pk2(0.f, 0.f);
         auto exps = [&](const uint32_t (&r)[32], uint32_t (&pk)[16]) {
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const float p0 = exp2f(fmaf(__uint_as_float(r[2 * i]), scale_log2, neg_m));
-            const float p1 = exp2f(fmaf(__uint_as_float(r[2 * i + 1]), scale_log2, neg_m));
-            sum0 += p0;
-            sum1 += p1;
+            const uint64_t x2 = fma2(pk2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1])), scale2, neg_m2);
+            float p0, p1;
+            if (i >= 16 - kPolyPairs) {
+              exp2_pair_fma(x2, p0, p1);
+            } else {
+              float x0, x1;
+              unpk2(x2, x0, x1);
+              p0 = ex2_approx(x0);
+              p1 = ex2_approx(x1);
+            }
+            sum2 = add2(sum2, pk2(p0, p1));
             pk[i] = pack2(p0, p1);
           }
         };
@@ -420,11 +493,14 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
         store(pk1, 1);
         store(pk2, 2);
         store(pk3, 3);
-        l_sum += sum0 + sum1;
+        {
+          float sum0, sum1;
+          unpk2(sum2, sum0, sum1);
+          l_sum += sum0 + sum1;
+        }
         tc::tmem_st_wait();
         tc::tc_fence_before();
         tc::mbar_arrive(bar(B_P, t));
-        if (quarter == 0 && lane == 0) KV_ATRACE(t * 4 + 3, s);
       }
       if (!ok) break;
       // ---- epilogue of the item: O / l -> bf16 rows.  O is taken into registers in one go and handed back, so
@@ -440,7 +516,7 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
       tc::tc_fence_before();
       tc::mbar_arrive(bar(B_O_FREE, t));
       const float inv = 1.f / l_sum;
-      const int head = w.head_a + t;
+      const int head = t == 0 ? w.head_a : w.head_b;
       // A thread owns a row, and rows are n_q_heads * D * 2 bytes apart in memory: stored directly, every
       // instruction would touch 32 different lines.  Each 32-column slab therefore goes through a 2 KiB
       // shared-memory buffer of the warp (16-byte pieces XOR-swizzled by the row), and is written out with four
@@ -515,11 +591,12 @@ int gather_prefix_kv(bf16 *qkv_ctx, int pos0, int n_q_heads, int n_kv_heads, int
   return KV_OK;
 }
 
-// head_dim 64 or 128, even number of query heads per KV head.  qkv_ctx has pos0 + n_tokens rows (see the file
-// header); out has n_tokens rows.
+// head_dim 64 or 128.  qkv_ctx has pos0 + n_tokens rows (see the file header); out has n_tokens rows.
 int attention_prefill_tc(const bf16 *qkv_ctx, int n_tokens, int pos0, int n_q_heads, int n_kv_heads, int head_dim,
                          bf16 *out, int *status_dev, cudaStream_t st) {
   if (n_tokens <= 0) return KV_OK;
+  if ((head_dim != 64 && head_dim != 128) || n_kv_heads <= 0 || n_q_heads <= 0 || n_q_heads % n_kv_heads != 0)
+    return KV_ERR_SHAPE;
   const int qkv_dim = (n_q_heads + 2 * n_kv_heads) * head_dim;
   CUtensorMap map;
   int rc = tc::make_tmap_2d(&map, qkv_ctx, pos0 + n_tokens, qkv_dim, qkv_dim, kBM);
@@ -548,7 +625,7 @@ int attention_prefill_tc(const bf16 *qkv_ctx, int n_tokens, int pos0, int n_q_he
   }
   if (regs_ok_dev[device] != 1) return KV_ERR_SHAPE;
   const int m_tiles = (n_tokens + kBM - 1) / kBM;
-  const int items = m_tiles * (n_q_heads / 2);
+  const int items = m_tiles * n_kv_heads * ((n_q_heads / n_kv_heads + 1) / 2);
   const int sms = sm_count(device);
   const int grid = items < sms ? items : sms;      // persistent: one CTA per SM walks the items
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)head_dim);
@@ -563,11 +640,5 @@ int attention_prefill_tc(const bf16 *qkv_ctx, int n_tokens, int pos0, int n_q_he
   KV_CUDA(cudaGetLastError());
   return KV_OK;
 }
-
-#ifdef KV_ATTN_TRACE
-extern "C" int kv_debug_attn_trace(long long *out_host) {
-  return cudaMemcpyFromSymbol(out_host, g_attn_trace, sizeof(long long) * 64 * 32) == cudaSuccess ? 0 : -13;
-}
-#endif
 
 }  // namespace kvr

@@ -33,6 +33,20 @@ inline CacheView make_view(const kv_cache_desc *c) {
   return v;
 }
 
+// Host-side validation of a cache descriptor, shared by every entry point that takes one.
+inline int check_cache_desc(const kv_cache_desc *c) {
+  if (c == nullptr || c->base_dev == nullptr) return KV_ERR_ARG;
+  if (c->num_blocks <= 0 || c->block_size <= 0 || c->n_layers <= 0 || c->n_kv_heads <= 0 || c->head_dim <= 0)
+    return KV_ERR_ARG;
+  if (c->elem_bytes != 2) return KV_ERR_SHAPE;
+  const long long page = (long long)c->block_size * c->n_kv_heads * c->head_dim * 2;
+  if (page % 16 != 0) return KV_ERR_SHAPE;
+  if (((uintptr_t)c->base_dev & 15) || (c->layer_stride & 15) || (c->kv_stride & 15) || (c->block_stride & 15))
+    return KV_ERR_ARG;
+  if (c->block_stride < page || c->kv_stride <= 0 || c->layer_stride <= 0) return KV_ERR_ARG;
+  return KV_OK;
+}
+
 // Layout of the device status word block at the start of every prefill/decode workspace.
 struct DeviceStatus {
   int error;      // 0, or the code of the first bounded wait that ran out
@@ -91,24 +105,19 @@ int gemm_tc(const bf16 *a, int lda, const bf16 *w, int m, int n, int k, int mode
 // CTA-pair (cta_group::2) variant with 256 x 256 tiles; same contract
 int gemm_tc_pair(const bf16 *a, int lda, const bf16 *w, int m, int n, int k, int mode, bf16 *out, float *resid,
                  int *status_dev, cudaStream_t st, const QkvRopeArgs *qkv_args = nullptr);
-int gemm_simt(const bf16 *a, int lda, const bf16 *w, int m, int n, int k, int mode, bf16 *out,
-              float *resid, cudaStream_t st);
+// the tile width (columns of W per tile) the launchers above pick for an m x n_out problem on `sms` SMs
+int gemm_tc_tile_width(int m, int n_out, int sms, int mode, int head_dim);
+int gemm_tc_pair_tile_width(int m, int n_out, int sms, int mode, int head_dim);
 
 int embed_rows(const bf16 *embed, const int *ids_dev, int n_tokens, int hidden, float *x, cudaStream_t st);
 int rmsnorm_rows(const float *x, const bf16 *gain, int rows, int dim, float eps, bf16 *out, cudaStream_t st);
 // positions pos0 + t, or row_pos[t] when row_pos is given (rows of several requests)
 int rope_table(float2 *table, int pos0, int n_tokens, int head_dim, float base, cudaStream_t st,
                const int *row_pos = nullptr);
-inline bool attention_tc_supported(int n_q_heads, int n_kv_heads, int head_dim) {
-  return (head_dim == 64 || head_dim == 128) && ((n_q_heads / n_kv_heads) % 2 == 0);
-}
 int attention_prefill_tc(const bf16 *qkv_ctx, int n_tokens, int pos0, int n_q_heads, int n_kv_heads, int head_dim,
                          bf16 *out, int *status_dev, cudaStream_t st);
 int gather_prefix_kv(bf16 *qkv_ctx, int pos0, int n_q_heads, int n_kv_heads, int head_dim, CacheView cache, int layer,
                      const int *block_table_dev, cudaStream_t st);
-int attention_prefill(const bf16 *qkv, int n_tokens, int pos0, int n_q_heads, int n_kv_heads,
-                      int head_dim, CacheView cache, int layer, const int *block_table_dev, bf16 *out,
-                      int *status_dev, cudaStream_t st);
 
 // decode-step kernels (one token, fp32 activations)
 int embed_one(const bf16 *embed, int token, int hidden, float *x, cudaStream_t st);
@@ -124,10 +133,17 @@ long long paged_attention_scratch_bytes(int n_q_heads, int head_dim, int n_ctx);
 int paged_attention(const float *q, int n_q_heads, CacheView cache, int layer, const int *block_table_dev,
                     int n_ctx, void *scratch, float *out, cudaStream_t st);
 
-int copy_pages(CacheView cache, int n_layers, const int *ids_host, int n_blocks, char *wire,
-               int wire_layout, int total_blocks_in_wire, int first_block_in_wire, bool to_wire,
+// One request of a pack/unpack call: n_blocks physical ids (host array) and the request's wire buffer (device).
+struct CopyRequest {
+  const int *ids_host;
+  int n_blocks;
+  char *wire;
+};
+// Every page of every request in as few launches as the parameter block allows (one for up to 7,680 blocks
+// of up to 64 requests).
+int copy_pages(CacheView cache, int n_layers, const CopyRequest *reqs, int n_req, int wire_layout, bool to_wire,
                cudaStream_t st);
-int copy_wait_expired(cudaStream_t st);   // KV_ERR_DEVICE if a pack/unpack kernel gave up a wait
+int copy_wait_expired(cudaStream_t st);   // KV_ERR_DEVICE if a pack/unpack kernel gave up a wait since the last check
 int fill_pattern(void *dst, long long bytes, unsigned long long seed, long long offset, cudaStream_t st);
 
 }  // namespace kvr

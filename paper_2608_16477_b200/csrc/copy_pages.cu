@@ -1,40 +1,49 @@
-// Pack (paged cache -> contiguous wire buffer) and unpack (wire buffer -> pages): byte-exact page copies.
+// Pack (paged cache -> contiguous wire buffers) and unpack (wire buffers -> pages): byte-exact page copies.
 //
-// One launch moves every page of up to kMaxIds logical blocks: block ids travel in the kernel
-// parameter block, so no device-side staging of the id list and no extra copy precede the kernel.
+// One launch moves every page of every request of a call: the physical block ids and one small record per
+// request (its wire buffer and its slice of the id list) travel in the kernel parameter block, so no
+// device-side staging of the id list and no extra copy precede the kernel.  Two parameter-block sizes are
+// compiled: up to 896 ids / 8 requests (under 4 KiB, the single-request calls of the migration path) and up
+// to 7,680 ids / 64 requests (under the 32 KiB limit of the launch interface, the batched calls); longer
+// lists are split over several launches.
 // A page (block_size * n_kv_heads * head_dim bf16) is contiguous on both sides; it moves as 16 KiB
 // bulk copies (cp.async.bulk) through a shared-memory ring.  HBM-bound: 2 * page bytes of traffic
 // per page, nothing is re-read.
+#include <vector>
+
 #include "common.cuh"
 
 namespace kvr {
 
-constexpr int kMaxIds = 960;          // keeps the parameter block under 4 KiB
-#ifndef KV_COPY_PIECE
-#define KV_COPY_PIECE 16384
-#define KV_COPY_BUFS 8
-#define KV_COPY_LAG 4
-#define KV_COPY_CTAS 1
-#endif
-constexpr int kPieceBytes = KV_COPY_PIECE;   // bytes per bulk copy
-constexpr int kBufs = KV_COPY_BUFS;          // shared-memory ring: 128 KiB per CTA, one CTA per SM (measured best: ~128 KiB in flight per SM)
-constexpr int kLag = KV_COPY_LAG;            // stores left in flight before a slot is refilled (kBufs - kLag loads in flight)
+constexpr int kPieceBytes = 16384;    // bytes per bulk copy
+constexpr int kBufs = 8;              // shared-memory ring: 128 KiB per CTA, one CTA per SM (measured best: ~128 KiB in flight per SM)
+constexpr int kLag = 4;               // stores left in flight before a slot is refilled (kBufs - kLag loads in flight)
 constexpr int kCopyThreads = 32;
-constexpr int kCtasPerSm = KV_COPY_CTAS;
 constexpr long long kCopyWaitLimit = 2000000000ll;   // cycles (~1 s): far beyond any legitimate wait
 
+// One request (or one slice of a request) inside a launch: ids[first_id .. first_id + n_blocks) are its blocks, in
+// the order they occupy wire positions wire_first .. wire_first + n_blocks - 1 of a wire buffer of wire_total blocks.
+struct CopySegment {
+  char *wire;
+  int first_id, n_blocks, wire_first, wire_total;
+};
+
+template <int MAX_IDS, int MAX_SEGS>
 struct PageCopyParams {
   CacheView cache;
-  char *wire;
   int n_layers;
-  int n_blocks;              // blocks in this launch
+  int n_blocks;              // blocks in this launch (all segments)
+  int n_segs;
   int layout;                // KV_WIRE_BLOCK_MAJOR / KV_WIRE_LAYER_MAJOR
-  int total_blocks;          // blocks in the whole wire buffer (layer-major stride)
-  int first_block;           // index of this launch's first block inside the wire buffer
   int page_bytes;
   int pieces_per_page;       // ceil(page_bytes / kPieceBytes)
-  int ids[kMaxIds];
+  CopySegment segs[MAX_SEGS];
+  int ids[MAX_IDS];
 };
+typedef PageCopyParams<896, 8> SmallCopyParams;
+typedef PageCopyParams<7680, 64> LargeCopyParams;
+static_assert(sizeof(SmallCopyParams) <= 4096, "single-request parameter block must stay under 4 KiB");
+static_assert(sizeof(LargeCopyParams) <= 32764, "parameter block exceeds the launch interface's limit");
 
 // Set by a copy kernel whose bounded wait ran out (the kernel then stops copying and returns).
 __device__ int g_copy_wait_expired = 0;
@@ -62,8 +71,8 @@ __device__ __forceinline__ bool cp_wait(uint32_t bar, uint32_t parity) {
 // shared -> global (bulk group).  Neither the LSU nor registers touch the payload, so the achieved
 // bandwidth does not depend on the SM clock.  A slot is refilled once the store that read it has
 // finished reading (wait_group.read), which keeps kBufs - kLag loads and kLag stores in flight per CTA.
-template <bool TO_WIRE>
-__global__ void __launch_bounds__(kCopyThreads) copy_pages_kernel(const __grid_constant__ PageCopyParams p) {
+template <bool TO_WIRE, typename Params>
+__global__ void __launch_bounds__(kCopyThreads) copy_pages_kernel(const __grid_constant__ Params p) {
   extern __shared__ __align__(128) unsigned char ring[];
   __shared__ __align__(8) unsigned long long full[kBufs];
   if (threadIdx.x != 0) return;
@@ -77,30 +86,36 @@ __global__ void __launch_bounds__(kCopyThreads) copy_pages_kernel(const __grid_c
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 
-  auto locate = [&](long long k, const char *&src, char *&dst, uint32_t &bytes) {
+  // Items are visited in increasing order by the loads and, a few items behind, by the stores: each of the two
+  // walks keeps its own cursor into the segment list instead of searching it.
+  auto locate = [&](long long k, int &seg, const char *&src, char *&dst, uint32_t &bytes) {
     const long long item = blockIdx.x + k * gridDim.x;
     const long long pg = item / p.pieces_per_page;
     const int piece = (int)(item - pg * p.pieces_per_page);
-    const int i = (int)(pg / (2 * p.n_layers));
+    const int i = (int)(pg / (2 * p.n_layers));                      // block index inside the launch
     const int rem = (int)(pg - (long long)i * 2 * p.n_layers);
     const int layer = rem >> 1, kv = rem & 1;
+    while (seg + 1 < p.n_segs && i >= p.segs[seg].first_id + p.segs[seg].n_blocks) ++seg;
+    const CopySegment &sg = p.segs[seg];
+    const int w = sg.wire_first + (i - sg.first_id);                 // block position inside the request's wire
     long long wire_page;
     if (p.layout == KV_WIRE_BLOCK_MAJOR)
-      wire_page = ((long long)(p.first_block + i) * p.n_layers + layer) * 2 + kv;
+      wire_page = ((long long)w * p.n_layers + layer) * 2 + kv;
     else
-      wire_page = ((long long)layer * 2 + kv) * p.total_blocks + p.first_block + i;
+      wire_page = ((long long)layer * 2 + kv) * sg.wire_total + w;
     const long long off = (long long)piece * kPieceBytes;
     char *c = p.cache.page(layer, kv, p.ids[i]) + off;
-    char *w = p.wire + wire_page * p.page_bytes + off;
-    src = TO_WIRE ? c : w;
-    dst = TO_WIRE ? w : c;
+    char *wp = sg.wire + wire_page * p.page_bytes + off;
+    src = TO_WIRE ? c : wp;
+    dst = TO_WIRE ? wp : c;
     const long long left = p.page_bytes - off;
     bytes = (uint32_t)(left < kPieceBytes ? left : kPieceBytes);
   };
+  int load_seg = 0, store_seg = 0;
   auto load = [&](long long k) {
     const int slot = (int)(k % kBufs);
     const char *src; char *dst; uint32_t bytes;
-    locate(k, src, dst, bytes);
+    locate(k, load_seg, src, dst, bytes);
     const uint32_t bar = cp_smem(&full[slot]);
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -113,7 +128,7 @@ __global__ void __launch_bounds__(kCopyThreads) copy_pages_kernel(const __grid_c
     const int slot = (int)(k % kBufs);
     if (!cp_wait(cp_smem(&full[slot]), (uint32_t)((k / kBufs) & 1))) break;
     const char *src; char *dst; uint32_t bytes;
-    locate(k, src, dst, bytes);
+    locate(k, store_seg, src, dst, bytes);
     asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
                  ::"l"(dst), "r"(cp_smem(ring + slot * kPieceBytes)), "r"(bytes) : "memory");
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
@@ -127,49 +142,104 @@ __global__ void __launch_bounds__(kCopyThreads) copy_pages_kernel(const __grid_c
   asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // all stores complete before the CTA exits
 }
 
-int copy_pages(CacheView cache, int n_layers, const int *ids_host, int n_blocks, char *wire, int wire_layout,
-               int total_blocks_in_wire, int first_block_in_wire, bool to_wire, cudaStream_t st) {
+namespace {
+
+template <typename Params>
+int launch_copy(const Params &p, bool to_wire, int sms, cudaStream_t st) {
+  const long long items = (long long)p.n_blocks * p.n_layers * 2 * p.pieces_per_page;
+  const int grid = (int)(items < sms ? items : sms);
+  if (to_wire)
+    copy_pages_kernel<true, Params><<<grid, kCopyThreads, kBufs * kPieceBytes, st>>>(p);
+  else
+    copy_pages_kernel<false, Params><<<grid, kCopyThreads, kBufs * kPieceBytes, st>>>(p);
+  KV_COUNT_LAUNCH();
+  KV_CUDA(cudaGetLastError());
+  return KV_OK;
+}
+
+// Fills parameter blocks of one size from the request list, starting a new launch whenever the ids or the
+// segment records of the current one are used up (a request may continue in the next launch).
+template <typename Params, int MAX_IDS, int MAX_SEGS>
+int copy_requests(const CacheView &cache, int n_layers, const CopyRequest *reqs, int n_req, int wire_layout, bool to_wire,
+                  int sms, cudaStream_t st) {
+  Params p;
+  auto reset = [&]() {
+    p.cache = cache;
+    p.n_layers = n_layers;
+    p.layout = wire_layout;
+    p.page_bytes = (int)cache.page_bytes();
+    p.pieces_per_page = (p.page_bytes + kPieceBytes - 1) / kPieceBytes;
+    p.n_blocks = 0;
+    p.n_segs = 0;
+  };
+  reset();
+  for (int r = 0; r < n_req; ++r) {
+    int done = 0;
+    while (done < reqs[r].n_blocks) {
+      if (p.n_blocks == MAX_IDS || p.n_segs == MAX_SEGS) {
+        int rc = launch_copy(p, to_wire, sms, st);
+        if (rc != KV_OK) return rc;
+        reset();
+      }
+      const int take = reqs[r].n_blocks - done < MAX_IDS - p.n_blocks ? reqs[r].n_blocks - done : MAX_IDS - p.n_blocks;
+      CopySegment &sg = p.segs[p.n_segs++];
+      sg.wire = reqs[r].wire;
+      sg.first_id = p.n_blocks;
+      sg.n_blocks = take;
+      sg.wire_first = done;
+      sg.wire_total = reqs[r].n_blocks;
+      for (int i = 0; i < take; ++i) p.ids[p.n_blocks + i] = reqs[r].ids_host[done + i];
+      p.n_blocks += take;
+      done += take;
+    }
+  }
+  if (p.n_blocks > 0) return launch_copy(p, to_wire, sms, st);
+  return KV_OK;
+}
+
+}  // namespace
+
+int copy_pages(CacheView cache, int n_layers, const CopyRequest *reqs, int n_req, int wire_layout, bool to_wire,
+               cudaStream_t st) {
   static bool attr_set[kMaxDevices] = {};
   const int device = current_device();
   if (device < 0) return KV_ERR_CUDA;
   if (!attr_set[device]) {
-    KV_CUDA(cudaFuncSetAttribute(copy_pages_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    KV_CUDA(cudaFuncSetAttribute(copy_pages_kernel<true, SmallCopyParams>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kBufs * kPieceBytes));
-    KV_CUDA(cudaFuncSetAttribute(copy_pages_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    KV_CUDA(cudaFuncSetAttribute(copy_pages_kernel<false, SmallCopyParams>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kBufs * kPieceBytes));
+    KV_CUDA(cudaFuncSetAttribute(copy_pages_kernel<true, LargeCopyParams>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kBufs * kPieceBytes));
+    KV_CUDA(cudaFuncSetAttribute(copy_pages_kernel<false, LargeCopyParams>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kBufs * kPieceBytes));
     attr_set[device] = true;
   }
   const int sms = sm_count(device);
-  for (int done = 0; done < n_blocks; done += kMaxIds) {
-    PageCopyParams p;
-    p.cache = cache;
-    p.wire = wire;
-    p.n_layers = n_layers;
-    p.n_blocks = (n_blocks - done < kMaxIds) ? n_blocks - done : kMaxIds;
-    p.layout = wire_layout;
-    p.total_blocks = total_blocks_in_wire;
-    p.first_block = first_block_in_wire + done;
-    p.page_bytes = (int)cache.page_bytes();
-    p.pieces_per_page = (p.page_bytes + kPieceBytes - 1) / kPieceBytes;
-    for (int i = 0; i < p.n_blocks; ++i) p.ids[i] = ids_host[done + i];
-    const long long items = (long long)p.n_blocks * n_layers * 2 * p.pieces_per_page;
-    const long long cap = (long long)sms * kCtasPerSm;
-    const int grid = (int)(items < cap ? items : cap);
-    if (to_wire)
-      copy_pages_kernel<true><<<grid, kCopyThreads, kBufs * kPieceBytes, st>>>(p);
-    else
-      copy_pages_kernel<false><<<grid, kCopyThreads, kBufs * kPieceBytes, st>>>(p);
-    KV_COUNT_LAUNCH();
-  KV_CUDA(cudaGetLastError());
+  long long total = 0;
+  int live = 0;
+  for (int r = 0; r < n_req; ++r) {
+    total += reqs[r].n_blocks;
+    live += reqs[r].n_blocks > 0 ? 1 : 0;
   }
-  return KV_OK;
+  if (total == 0) return KV_OK;
+  if (total <= 896 && live <= 8)
+    return copy_requests<SmallCopyParams, 896, 8>(cache, n_layers, reqs, n_req, wire_layout, to_wire, sms, st);
+  return copy_requests<LargeCopyParams, 7680, 64>(cache, n_layers, reqs, n_req, wire_layout, to_wire, sms, st);
 }
 
+// Reads the flag a copy kernel raises when one of its bounded waits ran out, and clears it, so that one expired
+// wait is reported once and later, healthy copies on the device are not blamed for it.
 int copy_wait_expired(cudaStream_t st) {
   int flag = 0;
   KV_CUDA(cudaStreamSynchronize(st));
   KV_CUDA(cudaMemcpyFromSymbol(&flag, g_copy_wait_expired, sizeof(int)));
-  return flag ? KV_ERR_DEVICE : KV_OK;
+  if (flag != 0) {
+    const int zero = 0;
+    KV_CUDA(cudaMemcpyToSymbol(g_copy_wait_expired, &zero, sizeof(int)));
+    return KV_ERR_DEVICE;
+  }
+  return KV_OK;
 }
 
 // Counter-based fill: word w = mix(seed + w); the host-side generator computes the same function.

@@ -43,14 +43,6 @@ struct TileCfg {
   static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + kEpiBytes;
 };
 
-#ifdef KV_GEMM_TRACE
-__device__ long long g_gemm_trace[64 * 8];
-#define KV_TRACE(slot, idx) \
-  do { if (blockIdx.x == 0 && (idx) < 64) g_gemm_trace[(idx) * 8 + (slot)] = clock64(); } while (0)
-#else
-#define KV_TRACE(slot, idx) do { } while (0)
-#endif
-
 enum WaitTag { TAG_EMPTY = 1, TAG_FULL = 2, TAG_TMEM_EMPTY = 3, TAG_TMEM_FULL = 4 };
 
 template <int MODE, int BN>
@@ -109,7 +101,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
         const int m0 = (tile % m_tiles) * BM;
         const int n0 = (tile / m_tiles) * kOutCols;
-        KV_TRACE(0, (tile - (int)blockIdx.x) / (int)gridDim.x);
         for (int kb = 0; kb < k_blocks; ++kb) {
           ok = tc::mbar_wait(empty_bar(stage), phase ^ 1, abort_flag, status, TAG_EMPTY);
           if (!ok) break;
@@ -143,10 +134,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local) {
         const int buf = local & 1;
         const uint32_t acc_phase = (local >> 1) & 1;
-        if (lane == 0) KV_TRACE(1, local);
         ok = wwait(tempty_bar(buf), acc_phase ^ 1, TAG_TMEM_EMPTY);
         if (!ok) break;
-        if (lane == 0) KV_TRACE(2, local);
         tc::tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * kTmemBufStride;
         for (int kb = 0; kb < k_blocks; ++kb) {
@@ -163,7 +152,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
           if (++stage == kStages) { stage = 0; phase ^= 1; }
         }
         if (ok) tc::umma_commit_warp(tfull_bar(buf));
-        if (lane == 0) KV_TRACE(3, local);
       }
     }
   } else {
@@ -176,11 +164,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
       const uint32_t acc_phase = (local >> 1) & 1;
       const int m0 = (tile % m_tiles) * BM;
       const int n0 = (tile / m_tiles) * kOutCols;
-      if (warp == 2 && lane == 0) KV_TRACE(4, local);
       ok = tc::mbar_wait(tfull_bar(buf), acc_phase, abort_flag, status, TAG_TMEM_FULL);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
-      if (warp == 2 && lane == 0) KV_TRACE(5, local);
       tc::tc_fence_after();
       const int row = m0 + quarter * 32 + lane;
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + buf * kTmemBufStride;
@@ -188,7 +174,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
                                    reinterpret_cast<float4 *>(smem_gen + kStages * kStageBytes + 256));
       tc::tc_fence_before();
       tc::mbar_arrive(tempty_bar(buf));
-      if (warp == 2 && lane == 0) KV_TRACE(6, local);
     }
   }
 
@@ -225,12 +210,6 @@ int launch_gemm(const CUtensorMap &ta, const CUtensorMap &tb, int m, int n, int 
 // M x N problem on `sms` SMs.  SwiGLU tiles hold a gate half and an up half, so a BN-wide tile yields BN / 2
 // output columns; QKV tiles must hold whole heads.
 int pick_bn(int m, int n_out, int sms, int mode, int head_dim) {
-  if (const char *e = getenv("KV_GEMM_BN")) {     // experiments: force one tile width where the mode allows it
-    const int bn = atoi(e);
-    const bool shape_ok = bn >= 128 && bn <= 256 && bn % 32 == 0 &&
-                          !(mode == GEMM_QKV_ROPE && (bn % head_dim) != 0) && !(mode == GEMM_SWIGLU && (bn % 64) != 0);
-    if (shape_ok) return bn;
-  }
   const int widths[5] = {256, 224, 192, 160, 128};
   const double eff[5] = {1.00, 1.00, 0.99, 0.96, 0.85};     // measured: narrower tiles re-read A more often and
                                                              // amortise the per-stage barrier work over fewer flops
@@ -254,6 +233,8 @@ int pick_bn(int m, int n_out, int sms, int mode, int head_dim) {
 
 }  // namespace
 
+int gemm_tc_tile_width(int m, int n_out, int sms, int mode, int head_dim) { return pick_bn(m, n_out, sms, mode, head_dim); }
+
 int gemm_tc(const bf16 *a, int lda, const bf16 *w, int m, int n, int k, int mode, bf16 *out, float *resid,
             int *status_dev, cudaStream_t st, const QkvRopeArgs *qkv_args) {
   if (m <= 0 || n <= 0 || k <= 0) return KV_OK;
@@ -266,7 +247,7 @@ int gemm_tc(const bf16 *a, int lda, const bf16 *w, int m, int n, int k, int mode
     if (n != (qa.n_q_heads + 2 * qa.n_kv_heads) * qa.head_dim) return KV_ERR_SHAPE;
   }
   if ((k % 8) != 0 || (lda % 8) != 0 || (n % 8) != 0) return KV_ERR_SHAPE;
-  if (((uintptr_t)a & 15) || ((uintptr_t)w & 15)) return KV_ERR_ARG;
+  if (((uintptr_t)a & 15) || ((uintptr_t)w & 15) || ((uintptr_t)out & 15) || ((uintptr_t)resid & 15)) return KV_ERR_ARG;
   const int sms = sm_count(current_device());
   const int bn = pick_bn(m, n, sms, mode, mode == GEMM_QKV_ROPE ? qa.head_dim : 0);
   CUtensorMap ta, tb;
@@ -297,11 +278,5 @@ int gemm_tc(const bf16 *a, int lda, const bf16 *w, int m, int n, int k, int mode
 #undef KV_GEMM_CASE
   return KV_ERR_ARG;
 }
-
-#ifdef KV_GEMM_TRACE
-extern "C" int kv_debug_gemm_trace(long long *out_host) {
-  return cudaMemcpyFromSymbol(out_host, g_gemm_trace, sizeof(long long) * 64 * 8) == cudaSuccess ? 0 : -13;
-}
-#endif
 
 }  // namespace kvr

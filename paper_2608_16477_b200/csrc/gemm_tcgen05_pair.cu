@@ -266,12 +266,6 @@ int launch_pair(const CUtensorMap &ta, const CUtensorMap &tb, int m, int n, int 
 
 // Tile width minimising waves x width / efficiency over the SM pairs (same model as the one-CTA kernel).
 int pick_bn_pair(int m, int n_out, int sms, int mode, int head_dim) {
-  if (const char *e = getenv("KV_GEMM_BN")) {     // experiments: force one tile width where the mode allows it
-    const int bn = atoi(e);
-    const bool shape_ok = bn >= 128 && bn <= 256 && bn % 32 == 0 &&
-                          !(mode == GEMM_QKV_ROPE && (bn % head_dim) != 0) && !(mode == GEMM_SWIGLU && (bn % 64) != 0);
-    if (shape_ok) return bn;
-  }
   const int widths[5] = {256, 224, 192, 160, 128};
   const double eff[5] = {1.00, 0.99, 0.98, 0.92, 0.78};     // measured per-column cost relative to 256-wide tiles
   const long long m_tiles = (m + 2 * BM - 1) / (2 * BM);
@@ -295,6 +289,10 @@ int pick_bn_pair(int m, int n_out, int sms, int mode, int head_dim) {
 
 }  // namespace
 
+int gemm_tc_pair_tile_width(int m, int n_out, int sms, int mode, int head_dim) {
+  return pick_bn_pair(m, n_out, sms, mode, head_dim);
+}
+
 // CTA-pair GEMM, 256 x BN tiles.  Same contract as gemm_tc.
 int gemm_tc_pair(const bf16 *a, int lda, const bf16 *w, int m, int n, int k, int mode, bf16 *out, float *resid,
                  int *status_dev, cudaStream_t st, const QkvRopeArgs *qkv_args) {
@@ -308,7 +306,7 @@ int gemm_tc_pair(const bf16 *a, int lda, const bf16 *w, int m, int n, int k, int
     if (n != (qa.n_q_heads + 2 * qa.n_kv_heads) * qa.head_dim) return KV_ERR_SHAPE;
   }
   if ((k % 8) != 0 || (lda % 8) != 0 || (n % 8) != 0) return KV_ERR_SHAPE;
-  if (((uintptr_t)a & 15) || ((uintptr_t)w & 15)) return KV_ERR_ARG;
+  if (((uintptr_t)a & 15) || ((uintptr_t)w & 15) || ((uintptr_t)out & 15) || ((uintptr_t)resid & 15)) return KV_ERR_ARG;
   const int sms = sm_count(current_device());
   const int bn = pick_bn_pair(m, n, sms, mode, mode == GEMM_QKV_ROPE ? qa.head_dim : 0);
   CUtensorMap ta, tb;

@@ -44,17 +44,20 @@ extern "C" int32_t kv_op_paged_attention_noalloc(const float *q_dev, int32_t n_q
                                                  int32_t layer, const int32_t *block_table_dev, int32_t n_ctx,
                                                  float *out_dev, void *stream) {
   using namespace kvr;
-  if (q_dev == nullptr || block_table_dev == nullptr || out_dev == nullptr || n_ctx <= 0 || n_q_heads <= 0 ||
-      cache == nullptr || cache->base_dev == nullptr)
+  if (q_dev == nullptr || block_table_dev == nullptr || out_dev == nullptr || n_ctx <= 0 || n_q_heads <= 0)
     return KV_ERR_ARG;
-  if (cache->num_blocks <= 0 || cache->block_size <= 0 || cache->n_kv_heads <= 0 || cache->elem_bytes != 2 ||
-      layer < 0 || layer >= cache->n_layers || n_q_heads % cache->n_kv_heads != 0 ||
+  if (((uintptr_t)q_dev & 7) || ((uintptr_t)out_dev & 3)) return KV_ERR_ARG;
+  // the same descriptor checks as kv_op_paged_attention (alignment of the base and of every stride included:
+  // the kernel reads pages with 16-byte copies)
+  int rc = check_cache_desc(cache);
+  if (rc != KV_OK) return rc;
+  if (layer < 0 || layer >= cache->n_layers || n_q_heads % cache->n_kv_heads != 0 ||
       (cache->head_dim != 64 && cache->head_dim != 128))
     return KV_ERR_SHAPE;
   // the fixed array bounds the context length: reject what does not fit instead of spilling past it
   if (paged_attention_scratch_bytes(n_q_heads, cache->head_dim, n_ctx) > kNoAllocScratchBytes) return KV_ERR_WORKSPACE;
   void *scratch = nullptr;
-  int rc = scratch_for_current_device(&scratch);
+  rc = scratch_for_current_device(&scratch);
   if (rc != KV_OK) return rc;
   // Every partial record the merge pass reads is written by the split pass of the same call, so nothing
   // left in the array by an earlier call is ever consumed and nothing needs clearing.

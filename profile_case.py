@@ -1,17 +1,22 @@
 """Runs ONE kernel of the hot path a few times at the benchmark's shapes, for profiler captures.
 
-  python -m paper_2608_16477_b200.profile_case gemm_gate_up [--tokens 4096] [--iters 3]
+  python profile_case.py gemm_gate_up [--tokens 4096] [--iters 3]
   cases: gemm_qkv, gemm_o, gemm_gate_up, gemm_down, attention, pack, unpack, decode_gemv, decode_attention, prefill_layer
 
 Inputs are synthetic and larger than L2 where the kernel is bandwidth-bound; a few GB at most are held on
 the device so a multi-pass capture stays short.  Prints the CUDA-event time per launch.
 """
 import argparse
+import os
 import sys
 
 import numpy as np
 
-import synth
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import synth  # noqa: E402
 
 
 def main():

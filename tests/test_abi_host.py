@@ -152,3 +152,64 @@ def test_prefill_and_decode_rejections(kv):
     assert _status(kv.kv_decode_step, M, cache, 5, 63, [3, 1, 4], logits, workspace=dws, stream=0) == O.ERR_TABLE_SHORT
     assert _status(kv.kv_decode_step, M, cache, s.vocab, 63, table, logits, workspace=dws, stream=0) == O.ERR_TOKEN_RANGE
     lib.kv_model_destroy(h)
+
+
+def test_single_kernel_entry_points_reject_misaligned_arguments(kv):
+    """Every vector access of the single-kernel entry points is guarded on the host: a misaligned pointer or
+    descriptor returns KV_ERR_ARG and nothing is launched (the addresses here are fake and never dereferenced)."""
+    from paper_2608_16477_b200.binding import CacheDesc
+    lib = kv.load()
+    s = synth.ModelShape("pa", n_layers=2, hidden=64, n_q_heads=8, n_kv_heads=2, head_dim=128, ffn=64, vocab=16)
+    good = _FakeCache(kv, s, 16)
+    page = synth.kv_page_bytes(s)
+    q, out, table = 0x7500000000, 0x7500100000, 0x7500200000
+    scratch = 0x7500300000
+    need = kv.kv_paged_attention_scratch_bytes(8, 128, 100)
+
+    def both(desc, q=q, out=out):
+        a = lib.kv_op_paged_attention(q, 8, C.byref(desc), 0, table, 100, scratch, need, out, 0)
+        b = lib.kv_op_paged_attention_noalloc(q, 8, C.byref(desc), 0, table, 100, out, 0)
+        return a, b
+    def desc(**kw):
+        f = dict(base_dev=0x7000000000, layer_stride=2 * 16 * page, kv_stride=16 * page, block_stride=page,
+                 num_blocks=16, block_size=16, n_layers=2, n_kv_heads=2, head_dim=128, elem_bytes=2)
+        f.update(kw)
+        return CacheDesc(*[f[n] for n, _ in CacheDesc._fields_])
+    for bad in (desc(base_dev=0x7000000008), desc(layer_stride=2 * 16 * page + 8), desc(kv_stride=16 * page + 4),
+                desc(block_stride=page + 2), desc(block_stride=page - 16), desc(num_blocks=0)):
+        assert both(bad) == (O.ERR_ARG, O.ERR_ARG)
+    assert both(desc(elem_bytes=4)) == (O.ERR_SHAPE, O.ERR_SHAPE)
+    assert both(desc(head_dim=96)) == (O.ERR_SHAPE, O.ERR_SHAPE)
+    assert both(good.desc, q=q + 4) == (O.ERR_ARG, O.ERR_ARG)            # q is read as float2
+    assert both(good.desc, out=out + 2) == (O.ERR_ARG, O.ERR_ARG)
+    assert lib.kv_op_paged_attention(q, 8, C.byref(good.desc), 0, table, 100, scratch, need - 1, out, 0) == O.ERR_WORKSPACE
+    # projections: bf16 output is stored as 16-byte vectors, the residual stream updated as float4
+    a, w, o, r = 0x7600000000, 0x7600100000, 0x7600200000, 0x7600300000
+    for pair in (0, 0x100):
+        assert lib.kv_op_gemm(a, 64, w, 32, 64, 64, 0 | pair, o + 8, None, None, 0) == O.ERR_ARG
+        assert lib.kv_op_gemm(a, 64, w, 32, 64, 64, 1 | pair, None, r + 4, None, 0) == O.ERR_ARG
+        assert lib.kv_op_gemm(a + 2, 64, w, 32, 64, 64, 0 | pair, o, None, None, 0) == O.ERR_ARG
+        assert lib.kv_op_gemm(a, 32, w, 32, 64, 64, 0 | pair, o, None, None, 0) == O.ERR_ARG      # lda < k
+        assert lib.kv_op_gemm(a, 64, w, 32, 0, 64, 0 | pair, o, None, None, 0) == O.ERR_ARG
+        assert lib.kv_op_gemm(a, 64, w, 32, 60, 64, 0 | pair, o, None, None, 0) == O.ERR_SHAPE    # n not a multiple of 8
+    # prefill attention: head_dim and head grouping
+    assert lib.kv_op_attention_prefill(a, 10, 0, 8, 2, 96, None, 0, None, o, None, 0) == O.ERR_SHAPE
+    assert lib.kv_op_attention_prefill(a, 10, 0, 7, 2, 128, None, 0, None, o, None, 0) == O.ERR_SHAPE
+    assert lib.kv_op_attention_prefill(a + 8, 10, 0, 8, 2, 128, None, 0, None, o, None, 0) == O.ERR_ARG
+    assert lib.kv_op_attention_prefill(a, 10, 8, 8, 2, 128, C.byref(good.desc), 0, table, o, None, 0) == O.ERR_SPLIT_UNALIGNED
+    assert lib.kv_op_attention_prefill(a, 10, 16, 8, 2, 128, None, 0, table, o, None, 0) == O.ERR_ARG
+
+
+def test_gemm_plan_query(kv):
+    """The launcher's choice is a pure function of the problem size and the SM count (148 assumed without a device)."""
+    pair, bn = kv.kv_gemm_plan(128, 5120, 1)
+    assert pair is False and bn in (128, 160, 192, 224, 256)
+    pair, bn = kv.kv_gemm_plan(4096, 10240, 3, head_dim=128)
+    assert pair is True and bn % 128 == 0
+    pair, bn = kv.kv_gemm_plan(4096, 25600, 2)
+    assert pair is True and bn % 64 == 0
+    from paper_2608_16477_b200 import KVError
+    with pytest.raises(KVError):
+        kv.kv_gemm_plan(4096, 10240, 3, head_dim=96)
+    with pytest.raises(KVError):
+        kv.kv_gemm_plan(0, 10240, 1)

@@ -8,19 +8,19 @@ hold at any size and (b) sampled outputs the oracle computes one by one:
     of a prefill over t[0..n];
   * pack/unpack: sampled pages of the 128 MiB wire and of the destination cache equal the host-generated
     counter pattern of the source pages, the merged table is the oracle's, untouched blocks stay zero.
-The 8B shape (36 layers, 1,024 + 256 tokens) is checked at FULL depth against the oracle.
+The 8B shape (36 layers, 1,024 + 256 tokens) is checked at FULL depth against the oracle, and the 32B shape at the
+benchmark's prefix and suffix lengths at reduced depth (two layers).
 """
 import numpy as np
 import pytest
 
 import synth
 from oracle import kv_oracle as O
-from tests.scenario import error_stats, oracle_reference, run_gpu_scenario
+from tests.scenario import (LockstepOracle, elementwise_ok, error_stats, exact_bound, oracle_floor,
+                            run_gpu_scenario, storage_bound)
 
 pytestmark = pytest.mark.gpu
 
-BF16_FLOOR = 3e-3          # layer 0: rounding of the normed input and of the stored K/V only (measured 2.3e-3)
-PER_LAYER_NOISE = 1.2e-2   # relative noise one layer of bf16-stored activations adds, in quadrature (measured ~8.7e-3)
 
 
 @pytest.fixture(scope="module")
@@ -75,15 +75,15 @@ def test_32b_full_depth_properties(kv):
     torch.cuda.synchronize()
     st = error_stats(lg_dec.cpu().numpy(), lg_pre.cpu().numpy())
     print("decode vs prefill logits at depth 64:", st)
-    # the decode path keeps fp32 activations, the prefill path stores them in bf16: the two differ by the bf16
-    # storage noise accumulated over 64 layers (about 0.6 % per layer in quadrature: measured 4.6 %)
-    assert st["rel_l2"] <= 1e-1, st
+    # the decode path keeps fp32 activations, the prefill path stores them in bf16: the two differ by at most the
+    # bf16 storage noise accumulated over 64 layers (the oracle-only floor of that depth; measured 4.6 %)
+    assert st["rel_l2"] <= exact_bound(s.n_layers), (st, exact_bound(s.n_layers))
     # the appended K/V row of the decode step equals the prefill's row for that position up to bf16 rounding
     # slot 0 of the block opened for position 4096 (int16 bit patterns viewed as bf16 values)
     ka = cache.pages([table[-1]])[0, :, :, : s.n_kv_heads * s.head_dim].contiguous().view(torch.bfloat16).float()
     kb = cache.pages([int(t2[-1])])[0, :, :, : s.n_kv_heads * s.head_dim].contiguous().view(torch.bfloat16).float()
     rel = (torch.linalg.norm(ka - kb) / torch.linalg.norm(kb)).item()
-    assert rel <= 1e-1, rel
+    assert rel <= exact_bound(s.n_layers), rel
 
 
 def test_32b_full_size_pack_unpack_sampled(kv):
@@ -121,32 +121,93 @@ def test_32b_full_size_pack_unpack_sampled(kv):
     assert torch.equal(got, wire)
 
 
-def test_8b_full_depth_against_oracle(kv):
-    """36 layers, prefix 512 + suffix 64: the whole scenario against the exact oracle at FULL depth.
+def _per_layer(got_k, got_v, ref_k, ref_v, lo=0, hi=None):
+    rows = []
+    for l in range(got_k.shape[0]):
+        rows.append((error_stats(got_k[l, lo:hi], ref_k[l, lo:hi])["rel_l2"], error_stats(got_v[l, lo:hi], ref_v[l, lo:hi])["rel_l2"]))
+    return rows
 
-    bf16 storage of activations adds about 0.6 % relative noise per layer, which accumulates in quadrature
-    along the residual stream, so the bound on layer l's K/V is 6e-3 * sqrt(l + 1) (the stated 1e-2 holds for
-    the first layers only; no two-byte pipeline can hold it at depth 36)."""
+
+def test_8b_full_depth_against_oracle(kv):
+    """The 8B-shaped configuration as written: 36 layers, prefix 1,024 + suffix 256, single request, at FULL depth.
+
+    The oracle advances in lockstep with the weight upload (exact definition over all 1,281 tokens; the same
+    function with bfloat16 storage points over the prefix).  Three claims per layer:
+      * against the exact oracle the K/V stay within 1.5 x the floor that the oracle alone shows for two-byte
+        storage at that depth (tests/golden/bf16_depth_curve_8b.txt; the stated 1e-2 wherever the floor allows it);
+      * against the storage-precision oracle the prefix K/V stay within the drift of two correct realisations;
+      * pack / unpack / assemble are bit-exact, as everywhere."""
     s = synth.SHAPES["8b"]
     s = synth.ModelShape(**{**s.__dict__, "vocab": 8192})
-    k, n = 512, 512 + 64
+    k, n = 1024, 1024 + 256
     ids = synth.token_ids(s, 0, n + 1)
-    res = run_gpu_scenario(kv, s, 0, ids, k, n, num_blocks=256)
+    lock = LockstepOracle(s, 0, ids).add("exact", n + 1).add("bf16", k, act_bf16=True, want_logits=False)
+    model = kv.Model(s, lock.head, lock.layers)
+    res = run_gpu_scenario(kv, s, 0, ids, k, n, num_blocks=256, model=model)
     assert np.array_equal(res["merged"], res["expected_merged"])
     want_wire = O.pack_blocks(res["src_img"], res["src_suffix_ids"])
     assert np.array_equal(res["wire"], want_wire.reshape(-1))
-    Kref, Vref, logits_ref = oracle_reference(s, 0, ids, mm_dtype=np.float32)
-    per_layer = []
-    for l in range(s.n_layers):
-        ek = error_stats(res["K"][l], Kref[l])["rel_l2"]
-        ev = error_stats(res["V"][l], Vref[l])["rel_l2"]
-        per_layer.append((round(ek, 5), round(ev, 5)))
+    for s_id, d_id in zip(res["src_suffix_ids"], res["dst_ids"]):
+        assert np.array_equal(res["tgt_after_unpack"][:, :, d_id], res["src_img"][:, :, s_id])
+    Kref, Vref, logits_ref = lock.result("exact")
+    Kb, Vb, _ = lock.result("bf16")
+    exact = _per_layer(res["K"], res["V"], Kref, Vref)
+    prefix = _per_layer(res["K"], res["V"], Kb, Vb, 0, k)
     lg = error_stats(res["logits"], logits_ref)
-    print("8b full depth vs exact oracle: per-layer (K, V) rel_l2:", per_layer, "logits:", lg)
-    for l, (ek, ev) in enumerate(per_layer):
-        bound = BF16_FLOOR if l == 0 else PER_LAYER_NOISE * np.sqrt(l)
-        assert ek <= bound and ev <= bound, (l, ek, ev, bound)
-    assert lg["rel_l2"] <= PER_LAYER_NOISE * np.sqrt(s.n_layers), lg
+    print("8b full depth, per-layer (K, V) rel_l2 vs exact:", [(round(a, 5), round(b, 5)) for a, b in exact])
+    print("8b full depth, prefix per-layer (K, V) rel_l2 vs bf16-storage oracle:", [(round(a, 5), round(b, 5)) for a, b in prefix])
+    print("8b full depth logits vs exact:", lg, "bound", exact_bound(s.n_layers))
+    floors = [oracle_floor(Kb, Vb, Kref, Vref, l) for l in range(s.n_layers)]
+    print("8b full depth, oracle floor (bf16-storage vs exact) on these inputs:", [round(f, 5) for f in floors])
+    for l in range(s.n_layers):
+        # both the golden curve (256 tokens) and the floor measured on these 1,024 prefix tokens must hold
+        assert max(exact[l]) <= exact_bound(l, floors[l]), (l, exact[l], floors[l])
+        assert max(exact[l]) <= exact_bound(l), (l, exact[l], exact_bound(l))
+        assert max(prefix[l]) <= storage_bound(l), (l, prefix[l], storage_bound(l))
+    assert lg["rel_l2"] <= exact_bound(s.n_layers), lg
+
+
+def test_32b_bench_launch_configuration_against_oracle(kv):
+    """The whole scenario at the benchmark's own launch configuration (32B shape, prefix 4,096 + suffix 512, pools of
+    4,096 blocks, fragmented ids) at reduced depth against the oracle.  The projections must run the instantiations the
+    benchmark runs: CTA pairs with 256-wide tiles for QKV and gate/up, 224-wide for the O and down projections
+    (K = 8,192 and 25,600)."""
+    s = synth.SHAPES["32b"].with_layers(2)
+    s = synth.ModelShape(**{**s.__dict__, "vocab": 4096})
+    prefix, suffix, pool = 4096, 512, 4096
+    n = prefix + suffix
+    assert kv.kv_gemm_plan(prefix, s.qkv_dim, 3, head_dim=s.head_dim) == (True, 256)
+    assert kv.kv_gemm_plan(prefix, s.hidden, 1) == (True, 224)
+    assert kv.kv_gemm_plan(prefix, s.ffn, 2) == (True, 256)
+    ids = synth.token_ids(s, 0, n + 1)
+    lock = LockstepOracle(s, 0, ids).add("exact", n + 1).add("bf16", prefix, act_bf16=True, want_logits=False)
+    model = kv.Model(s, lock.head, lock.layers)
+    res = run_gpu_scenario(kv, s, 0, ids, prefix, n, num_blocks=pool, model=model)
+    assert np.array_equal(res["merged"], res["expected_merged"])
+    want_wire = O.pack_blocks(res["src_img"], res["src_suffix_ids"])
+    assert np.array_equal(res["wire"], want_wire.reshape(-1))
+    for s_id, d_id in zip(res["src_suffix_ids"], res["dst_ids"]):
+        assert np.array_equal(res["tgt_after_unpack"][:, :, d_id], res["src_img"][:, :, s_id])
+    Kref, Vref, logits_ref = lock.result("exact")
+    Kb, Vb, _ = lock.result("bf16")
+    report = {}
+    for l in range(2):
+        # the floor of two-byte storage for THIS shape and context length, from the two oracle evaluations
+        floor = oracle_floor(Kb, Vb, Kref, Vref, l)
+        report[f"oracle_floor{l}"] = floor
+        for nm, got, ref, refb in (("K", res["K"][l], Kref[l], Kb[l]), ("V", res["V"][l], Vref[l], Vb[l])):
+            st = error_stats(got, ref)
+            report[f"exact_{nm}{l}"] = st
+            bound = exact_bound(l, floor)
+            assert st["rel_l2"] <= bound and elementwise_ok(got, ref, bound), (l, nm, st, floor, bound)
+            sb = error_stats(got[:prefix], refb)
+            report[f"storage_{nm}{l}"] = sb
+            assert sb["rel_l2"] <= storage_bound(l), (l, nm, sb)
+            rms = float(np.sqrt(np.mean(np.asarray(refb, dtype=np.float64) ** 2)))
+            assert np.all(np.abs(got[:prefix] - refb) <= 8 * storage_bound(l) * rms + 2.0 ** -7 * np.abs(refb)), (l, nm, sb)
+    report["logits"] = error_stats(res["logits"], logits_ref)
+    print("32b x 2 layers at 4096 + 512:", report)
+    assert report["logits"]["rel_l2"] <= exact_bound(2), report["logits"]
 
 
 def test_pack_unpack_stress_16_requests_full_size(kv):
