@@ -127,6 +127,13 @@ int32_t kv_check_device_status(const void *workspace_dev, void *stream);
  * cleared by the call.  KV_OK otherwise. */
 int32_t kv_check_copy_status(void *stream);
 
+/* Self-test of the kernels' bounded waits (no counterpart in the paper; failure detection of this library): launches
+ * one small kernel whose threads wait, with the routine every tensor-core kernel uses, on a barrier that nothing
+ * signals.  The wait gives up after about limit_us microseconds (1..100000), records itself in the status block at
+ * status_dev (>= 32 bytes, 16-byte aligned; a prefill/decode workspace will do) and the kernel returns normally; a
+ * following kv_check_device_status(status_dev, stream) must report KV_ERR_DEVICE.  The GPU context stays usable. */
+int32_t kv_selftest_bounded_wait(void *status_dev, int32_t limit_us, void *stream);
+
 /* ---------------------------------------------------------------- the four operations */
 
 /* Target-side prefix reconstruction (Section 4.3 / Section 5: the target reconstructs the prefix KV

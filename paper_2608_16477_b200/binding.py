@@ -21,6 +21,7 @@ EXPORTS = [
     "kv_op_attention_prefill", "kv_paged_attention_scratch_bytes", "kv_op_paged_attention", "kv_fill_pattern",
     "kv_profile_enable", "kv_profile_read", "kv_launch_count", "kv_op_paged_attention_noalloc", "kv_check_copy_status", "kv_op_gemv",
     "kv_window_evaluate", "kv_window_select", "kv_window_waste_bound", "kv_ewma", "kv_prefill_prefix_batched",
+    "kv_selftest_bounded_wait",
 ]
 
 PROFILE_KINDS = ("embed", "rmsnorm", "gemm_qkv", "rope_store", "attention", "gemm_o", "gemm_gate_up", "gemm_down",
@@ -109,6 +110,7 @@ def load(build_if_missing: bool = True):
         "kv_fill_pattern": (i32, [vp, i64, C.c_uint64, i64, vp]),
         "kv_op_paged_attention_noalloc": (i32, [vp, i32, C.POINTER(CacheDesc), i32, vp, i32, vp, vp]),
         "kv_check_copy_status": (i32, [vp]),
+        "kv_selftest_bounded_wait": (i32, [vp, i32, vp]),
         "kv_window_evaluate": (i32, [C.POINTER(WindowInputs), C.c_double, C.POINTER(WindowEval)]),
         "kv_window_select": (i32, [C.POINTER(WindowInputs), C.c_double, C.c_double, C.POINTER(WindowEval),
                                    C.POINTER(C.c_int32)]),
@@ -395,6 +397,11 @@ def kv_op_paged_attention_noalloc(q, cache: PagedCache, layer, block_table_dev, 
     _check(load().kv_op_paged_attention_noalloc(_ptr(q), q.shape[0], C.byref(cache.desc), layer,
                                                 _ptr(block_table_dev), n_ctx, _ptr(out), _stream(stream)),
            "kv_op_paged_attention_noalloc")
+
+
+def kv_selftest_bounded_wait(status_buf, limit_us: int = 200, stream=None) -> None:
+    """Launches the bounded-wait self-test into `status_buf`; kv_check_device_status(status_buf) then raises KVError(-14)."""
+    _check(load().kv_selftest_bounded_wait(_ptr(status_buf), limit_us, _stream(stream)), "kv_selftest_bounded_wait")
 
 
 def kv_check_copy_status(stream=None) -> None:

@@ -127,6 +127,31 @@ int make_tmap_2d(CUtensorMap *map, const void *base, long long rows, long long c
 
 using namespace kvr;
 
+// Self-test of the bounded-wait machinery every tensor-core kernel relies on: thread 0 waits, with the kernels' own
+// wait routine and a short limit, on an mbarrier that nothing ever arrives on.  The wait must give up, record itself in
+// the status block and raise the CTA's abort flag; the second warp, waiting on the same barrier, must leave through
+// that flag without recording anything; the kernel then returns normally.  detail[3] = number of threads whose wait
+// reported failure (64 when everything works).
+constexpr int kTagSelfTest = 99;
+__global__ void bounded_wait_selftest_kernel(DeviceStatus *status, long long limit_cycles) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ int abort_flag;
+  __shared__ int gave_up;
+  if (threadIdx.x == 0) {
+    tc::mbar_init(tc::smem_u32(&bar), 1);
+    abort_flag = 0;
+    gave_up = 0;
+    tc::fence_barrier_init();
+  }
+  __syncthreads();
+  // thread 0 carries the short limit; everybody else would wait for the full ~1 s and must be released by the flag
+  const bool ok = tc::mbar_wait(tc::smem_u32(&bar), 0, &abort_flag, status, kTagSelfTest,
+                                threadIdx.x == 0 ? limit_cycles : tc::kWaitLimitCycles);
+  if (!ok) atomicAdd(&gave_up, 1);
+  __syncthreads();
+  if (threadIdx.x == 0) status->detail[3] = gave_up;
+}
+
 struct kv_model {
   kv_model_desc d;
   const bf16 *embed, *lm_head, *final_norm;
@@ -695,6 +720,16 @@ int32_t kv_op_paged_attention(const float *q_dev, int32_t n_q_heads, const kv_ca
 }
 
 int32_t kv_check_copy_status(void *stream) { return copy_wait_expired((cudaStream_t)stream); }
+
+int32_t kv_selftest_bounded_wait(void *status_dev, int32_t limit_us, void *stream) {
+  if (status_dev == nullptr || ((uintptr_t)status_dev & 15) || limit_us <= 0 || limit_us > 100000) return KV_ERR_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  KV_CUDA(cudaMemsetAsync(status_dev, 0, sizeof(DeviceStatus), st));
+  bounded_wait_selftest_kernel<<<1, 64, 0, st>>>(reinterpret_cast<DeviceStatus *>(status_dev), (long long)limit_us * 2000ll);
+  KV_COUNT_LAUNCH();
+  KV_CUDA(cudaGetLastError());
+  return KV_OK;
+}
 
 int32_t kv_profile_enable(int32_t on) {
   g_prof_on = on != 0;

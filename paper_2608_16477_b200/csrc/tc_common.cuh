@@ -46,14 +46,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // (it then records `tag` in the device status and raises the CTA-wide abort flag) or another thread
 // of the CTA already raised the flag.  Callers leave their loops on false; nothing spins forever.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                          DeviceStatus *status, int tag) {
+                                          DeviceStatus *status, int tag, long long limit_cycles = kWaitLimitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 0xff) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitLimitCycles) {
+      if (clock64() - t0 > limit_cycles) {
         *abort_flag = 1;
         if (status != nullptr && atomicCAS(&status->error, 0, KV_ERR_DEVICE) == 0) {
           status->where = tag;

@@ -466,3 +466,26 @@ def test_batched_prefill_equals_separate_calls(kv, torch, name, layers, lengths)
     kv.kv_prefill_prefix_batched(model, three, ids, tables)
     torch.cuda.synchronize()
     assert torch.equal(one.data, three.data)
+
+
+# ------------------------------------------------------------------ failure detection on the device
+def test_bounded_wait_gives_up_and_reports(kv, torch):
+    """Every wait inside the tensor-core kernels is bounded.  The self-test kernel makes one run out on purpose (a
+    barrier that nothing signals, a 200 us limit): the wait records itself in the status block, the other threads
+    leave through the CTA's abort flag, the kernel returns, the host reads KV_ERR_DEVICE, and the context is intact:
+    the next operation on the same workspace runs and reports a clean status."""
+    s = synth.SHAPES["tiny"]
+    head = synth.head_weights(s, 0)
+    model = kv.Model(s, head, lambda l: synth.layer_weights(s, 0, l))
+    ws = model.workspace(kv.KV_OP_PREFILL, 64)
+    kv.kv_selftest_bounded_wait(ws, 200)
+    with pytest.raises(kv.KVError) as e:
+        kv.kv_check_device_status(ws)
+    assert e.value.status == -14                                   # KV_ERR_DEVICE
+    words = ws[:32].view(torch.int32).tolist()                     # error, tag, detail[0..5]
+    assert words[0] == -14 and words[1] == 99 and words[2] == 0 and words[3] == 0
+    assert words[5] == 64                                          # every thread's wait was abandoned, one recorded
+    cache = kv.PagedCache(s, 16, fill=0)
+    kv.kv_prefill_prefix(model, cache, synth.token_ids(s, 0, 64), [3, 1, 4, 5], workspace=ws)
+    kv.kv_check_device_status(ws)                                  # clean again
+    assert bool(cache.data.any())
