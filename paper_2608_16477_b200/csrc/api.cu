@@ -206,6 +206,7 @@ PrefillWs carve_prefill(const kv_model_desc &d, void *base, int max_tokens, int 
 struct DecodeWs {
   DeviceStatus *status;
   int *table;
+  float2 *rope;
   float *x, *h, *qkv, *o, *mid;
   void *scratch;
   long long bytes;
@@ -217,6 +218,7 @@ DecodeWs carve_decode(const kv_model_desc &d, void *base, int max_ctx, int block
   const long long qkv_dim = (long long)(d.n_q_heads + 2 * d.n_kv_heads) * d.head_dim;
   w.status = c.take<DeviceStatus>(1);
   w.table = c.take<int>((max_ctx + block_size - 1) / block_size + 1);
+  w.rope = c.take<float2>(d.head_dim / 2);
   w.x = c.take<float>(d.hidden);
   w.h = c.take<float>(d.hidden);
   w.qkv = c.take<float>(qkv_dim);
@@ -527,9 +529,13 @@ int32_t kv_decode_step(kv_model *m, const kv_cache_desc *cache, int32_t token_id
 
   KV_CUDA(cudaMemsetAsync(w.status, 0, sizeof(DeviceStatus), st));
   KV_CUDA(cudaMemcpyAsync(w.table, block_table_host, sizeof(int) * need_blocks, cudaMemcpyHostToDevice, st));
-  { ProfScope ps(PROF_DECODE_OTHER, st); KV_TRY(embed_one(m->embed, token_id, d.hidden, w.x, st)); }
+  {
+    ProfScope ps(PROF_DECODE_OTHER, st);
+    KV_TRY(rope_table(w.rope, pos, 1, d.head_dim, d.rope_base, st));
+    KV_TRY(embed_one(m->embed, token_id, d.hidden, w.x, st));
+  }
   for (int l = 0; l < d.n_layers; ++l) {
-    { ProfScope ps(PROF_DECODE_GEMV, st); KV_TRY(gemv_qkv_rope(m->w_qkv[l], w.x, m->attn_norm[l], d.rms_eps, d.hidden, pos, d.n_q_heads, d.n_kv_heads, d.head_dim, d.rope_base, cv, l, w.table, w.qkv, st)); }
+    { ProfScope ps(PROF_DECODE_GEMV, st); KV_TRY(gemv_qkv_rope(m->w_qkv[l], w.x, m->attn_norm[l], d.rms_eps, d.hidden, pos, d.n_q_heads, d.n_kv_heads, d.head_dim, w.rope, cv, l, w.table, w.qkv, st)); }
     { ProfScope ps(PROF_DECODE_ATTENTION, st); KV_TRY(paged_attention(w.qkv, d.n_q_heads, cv, l, w.table, n_ctx, w.scratch, w.o, st)); }
     { ProfScope ps(PROF_DECODE_GEMV, st); KV_TRY(gemv(m->w_o[l], w.o, d.hidden, q_dim, 1, w.x, st)); }
     { ProfScope ps(PROF_DECODE_GEMV, st); KV_TRY(gemv(m->w_gate_up[l], w.x, d.ffn, d.hidden, 2, w.mid, st, m->ffn_norm[l], d.rms_eps)); }

@@ -125,10 +125,11 @@ int embed_one(const bf16 *embed, int token, int hidden, float *x, cudaStream_t s
 // gain != nullptr fuses RMSNorm(x, gain, eps) into the product (modes 0 and 2)
 int gemv(const bf16 *w, const float *x, int n, int k, int mode, float *y, cudaStream_t st,
          const bf16 *gain = nullptr, float eps = 0.f);
-// RMSNorm + QKV projection + RoPE + K/V append of one decode token; q_out = rotated fp32 queries
+// RMSNorm + QKV projection + RoPE + K/V append of one decode token; q_out = rotated fp32 queries;
+// rope_dev: (cos, sin) of position `pos` for the head_dim / 2 frequencies (rope_table with one token)
 int gemv_qkv_rope(const bf16 *w_qkv, const float *x, const bf16 *gain, float eps, int hidden, int pos, int n_q_heads,
-                  int n_kv_heads, int head_dim, float base, CacheView cache, int layer, const int *block_table_dev,
-                  float *q_out, cudaStream_t st);
+                  int n_kv_heads, int head_dim, const float2 *rope_dev, CacheView cache, int layer,
+                  const int *block_table_dev, float *q_out, cudaStream_t st);
 long long paged_attention_scratch_bytes(int n_q_heads, int head_dim, int n_ctx);
 int paged_attention(const float *q, int n_q_heads, CacheView cache, int layer, const int *block_table_dev,
                     int n_ctx, void *scratch, float *out, cudaStream_t st);

@@ -40,16 +40,16 @@ __device__ __forceinline__ float dot8(uint4 wraw, float4 x0, float4 x1) {
 // NORM fuses the preceding RMSNorm: the warp accumulates sum(x^2) from the values it loads anyway and
 // computes W . (x * gain) * rsqrt(mean(x^2) + eps), so no separate normalisation launch is needed.
 // Epilogues: STORE rows (2u, 2u+1); ADD into the residual; SWIGLU rows (u, u + n) -> silu(a) * b;
-// QKV rows (j, j + d/2) of one head -> RoPE rotation, q to the fp32 query vector, k and v (bf16) appended
-// to the paged cache.
+// QKV rows (j, j + d/2) of one head -> RoPE rotation (cos/sin of the step's position from a table built once per
+// step with fp64 angles), q to the fp32 query vector, k and v (bf16) appended to the paged cache.
 enum GemvEpi { GEMV_STORE = 0, GEMV_ADD = 1, GEMV_SWIGLU = 2, GEMV_QKV = 3 };
 constexpr int kGemvWarps = 8;
 
 struct GemvQkvArgs {
   CacheView cache;
   const int *block_table;
+  const float2 *rope;       // (cos, sin) of the step's position for each of the head_dim / 2 frequencies
   int pos, layer, head_dim, n_q_heads, n_kv_heads;
-  float base;
 };
 
 template <int EPI, bool NORM>
@@ -148,10 +148,9 @@ __global__ void __launch_bounds__(kGemvWarps * 32) gemv2_kernel(const bf16 *__re
     const int block = qa.block_table[qa.pos / qa.cache.block_size];
     const long long slot_off = (long long)(qa.pos % qa.cache.block_size) * qa.n_kv_heads * d;
     if (head < qa.n_q_heads + qa.n_kv_heads) {
-      double sn, cs;
-      sincos((double)qa.pos * pow((double)qa.base, -(double)j / (double)half), &sn, &cs);
-      const float ra = acc_a * (float)cs - acc_b * (float)sn;
-      const float rb = acc_b * (float)cs + acc_a * (float)sn;
+      const float2 cs = qa.rope[j];
+      const float ra = acc_a * cs.x - acc_b * cs.y;
+      const float rb = acc_b * cs.x + acc_a * cs.y;
       if (head < qa.n_q_heads) {
         y[row_a] = ra;
         y[row_b] = rb;
@@ -203,8 +202,8 @@ int gemv(const bf16 *w, const float *x, int n, int k, int mode, float *y, cudaSt
 // Fused decode-step front end of a layer: RMSNorm + QKV projection + RoPE + K/V append.
 // q_out receives the rotated fp32 query vector [n_q_heads * head_dim].
 int gemv_qkv_rope(const bf16 *w_qkv, const float *x, const bf16 *gain, float eps, int hidden, int pos, int n_q_heads,
-                  int n_kv_heads, int head_dim, float base, CacheView cache, int layer, const int *block_table_dev,
-                  float *q_out, cudaStream_t st) {
+                  int n_kv_heads, int head_dim, const float2 *rope_dev, CacheView cache, int layer,
+                  const int *block_table_dev, float *q_out, cudaStream_t st) {
   GemvQkvArgs qa;
   qa.cache = cache;
   qa.block_table = block_table_dev;
@@ -213,7 +212,7 @@ int gemv_qkv_rope(const bf16 *w_qkv, const float *x, const bf16 *gain, float eps
   qa.head_dim = head_dim;
   qa.n_q_heads = n_q_heads;
   qa.n_kv_heads = n_kv_heads;
-  qa.base = base;
+  qa.rope = rope_dev;
   if (hidden % 8 != 0) return KV_ERR_SHAPE;
   const int n = (n_q_heads + 2 * n_kv_heads) * head_dim;
   return launch_gemv2<GEMV_QKV, true>(w_qkv, x, gain, eps, n, hidden, q_out, qa, st);

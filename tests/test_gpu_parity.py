@@ -175,7 +175,9 @@ def test_gemm_cta_pair_identical_to_single_cta(kv, torch, m, n, k, mode):
     assert bool(res[0].float().abs().sum() > 0)
 
 
-@pytest.mark.parametrize("n,k", [(37, 256), (512, 5120), (1001, 1064)])
+# (14400, 64): enough row pairs to fill the SMs with warps (the lighter four-loads-in-flight form of the kernel);
+# the other cases run the form with eight loads in flight per row and lane
+@pytest.mark.parametrize("n,k", [(37, 256), (512, 5120), (1001, 1064), (14400, 64), (300, 2056)])
 @pytest.mark.parametrize("mode,norm", [(0, False), (0, True), (1, False), (2, False), (2, True)])
 def test_gemv_decode(kv, torch, n, k, mode, norm):
     rng = np.random.default_rng(n + k + mode)
