@@ -1,7 +1,8 @@
 """Runs ONE kernel of the hot path a few times at the benchmark's shapes, for profiler captures.
 
   python profile_case.py gemm_gate_up [--tokens 4096] [--iters 3]
-  cases: gemm_qkv, gemm_o, gemm_gate_up, gemm_down, attention, pack, unpack, decode_gemv, decode_attention, prefill_layer
+  cases: gemm_qkv, gemm_o, gemm_gate_up, gemm_down, attention, pack, unpack, pack_batched, unpack_batched, decode_gemv,
+         decode_gemv_o, decode_attention, prefill_layer
 
 Inputs are synthetic and larger than L2 where the kernel is bandwidth-bound; a few GB at most are held on
 the device so a multi-pass capture stays short.  Prints the CUDA-event time per launch.
@@ -84,6 +85,40 @@ def main():
             else:
                 kv.kv_unpack_assemble(cache, wires[i], np.arange(a.blocks), ids, [], a.blocks * s.block_size)
         work, unit = 2.0 * a.blocks * s.n_layers * 2 * cache.page_bytes / 1e9, "GB/s"
+    elif a.case in ("pack_batched", "unpack_batched"):
+        # the 16-request stress workload at 1/16 of its block counts (289 blocks, 1.1 GiB payload) in the batched form:
+        # one launch for all requests
+        pool = 1024
+        cache = kv.PagedCache(s, pool)
+        kv.kv_fill_pattern(cache.data, cache.data.numel() * 2, seed=1)
+        counts = [max(1, c // 16) for c in synth.STRESS_BLOCK_COUNTS]
+        offs = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+        n_sets = 2
+        perms = [synth.block_permutation(1 + i, pool)[: offs[-1]] for i in range(n_sets)]
+        block_bytes = s.n_layers * 2 * cache.page_bytes
+        wires = [[torch.empty(c * block_bytes, dtype=torch.uint8, device=dev) for c in counts] for _ in range(n_sets)]
+        state = {"i": 0}
+
+        def run():
+            i = state["i"] % n_sets
+            state["i"] += 1
+            if a.case == "pack_batched":
+                kv.kv_pack_blocks_batched(cache, offs, perms[i], wires[i])
+            else:
+                kv.kv_unpack_blocks_batched(cache, offs, perms[i], wires[i])
+        work, unit = 2.0 * int(offs[-1]) * block_bytes / 1e9, "GB/s"
+    elif a.case == "decode_gemv_o":
+        # the O projection of one decode step (5120 x 8192, 84 MB: a SHORT launch), residual-add epilogue, rotating over
+        # 6 weight copies (> L2)
+        ws = [rnd(s.hidden, s.q_dim, std=0.02) for _ in range(6)]
+        x = torch.randn(s.q_dim, device=dev)
+        y = torch.zeros(s.hidden, device=dev)
+        state = {"i": 0}
+
+        def run():
+            state["i"] += 1
+            kv.kv_op_gemv(ws[state["i"] % 6], x, 1, y)
+        work, unit = ws[0].numel() * 2 / 1e9, "GB/s"
     elif a.case == "decode_gemv":
         # the gate/up product of one decode step (524 MB of weights), rotating over 4 weight copies (> L2)
         ws = [rnd(2 * s.ffn, s.hidden, std=0.02) for _ in range(4)]
