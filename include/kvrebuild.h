@@ -111,6 +111,15 @@ int32_t kv_model_destroy(kv_model *m);
  * The workspace must be 1024-byte aligned. */
 int64_t kv_workspace_bytes(const kv_model *m, int32_t op, int32_t max_tokens);
 
+/* Where the residual stream (the hidden state x, fp32) sits inside a workspace of kv_workspace_bytes(m, op, max_tokens)
+ * bytes: *offset_out bytes from its base, *bytes_out long (KV_OP_PREFILL: [max_tokens, hidden] rows of the call's
+ * tokens; KV_OP_DECODE: [hidden]).  After a call it holds the output of the last layer that ran: for a K/V-only
+ * prefill (logits_out_dev = NULL) that is the INPUT of the model's last layer, whose K/V depend on nothing else.  Lets a
+ * caller read hidden states, and lets a test check any single layer of a deep model against the oracle on that
+ * layer's true input. */
+int32_t kv_workspace_residual(const kv_model *m, int32_t op, int32_t max_tokens, int64_t *offset_out,
+                              int64_t *bytes_out);
+
 const char *kv_status_string(int32_t status);
 /* Text of the last CUDA error seen by this thread's calls ("" if none). */
 const char *kv_last_cuda_error(void);

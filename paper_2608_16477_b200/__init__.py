@@ -6,7 +6,7 @@ shared library is missing and cannot be built.
 """
 from .binding import (KVError, load, lib_path, status_string, Model, PagedCache, kv_bytes_per_token,
                       kv_prefill_prefix, kv_prefill_prefix_batched, kv_pack_blocks, kv_unpack_assemble, kv_decode_step,
-                      kv_pack_blocks_batched, kv_unpack_blocks_batched, kv_workspace_bytes,
+                      kv_pack_blocks_batched, kv_unpack_blocks_batched, kv_workspace_bytes, kv_workspace_residual,
                       kv_check_device_status, kv_check_copy_status, kv_selftest_bounded_wait, kv_window_evaluate, kv_window_select,
                       kv_window_waste_bound, kv_ewma, kv_op_gemm, kv_gemm_plan, kv_op_gemv, kv_op_rmsnorm,
                       kv_op_attention_prefill, kv_op_paged_attention, kv_op_paged_attention_noalloc, kv_paged_attention_scratch_bytes,

@@ -21,7 +21,7 @@ EXPORTS = [
     "kv_op_attention_prefill", "kv_paged_attention_scratch_bytes", "kv_op_paged_attention", "kv_fill_pattern",
     "kv_profile_enable", "kv_profile_read", "kv_launch_count", "kv_op_paged_attention_noalloc", "kv_check_copy_status", "kv_op_gemv",
     "kv_window_evaluate", "kv_window_select", "kv_window_waste_bound", "kv_ewma", "kv_prefill_prefix_batched",
-    "kv_selftest_bounded_wait",
+    "kv_selftest_bounded_wait", "kv_workspace_residual",
 ]
 
 PROFILE_KINDS = ("embed", "rmsnorm", "gemm_qkv", "rope_store", "attention", "gemm_o", "gemm_gate_up", "gemm_down",
@@ -89,6 +89,7 @@ def load(build_if_missing: bool = True):
         "kv_model_create": (i32, [C.POINTER(ModelDesc), C.POINTER(Weights), C.POINTER(vp)]),
         "kv_model_destroy": (i32, [vp]),
         "kv_workspace_bytes": (i64, [vp, i32, i32]),
+        "kv_workspace_residual": (i32, [vp, i32, i32, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]),
         "kv_status_string": (C.c_char_p, [i32]),
         "kv_last_cuda_error": (C.c_char_p, []),
         "kv_bytes_per_token": (i64, [i32, i32, i32, i32]),
@@ -257,6 +258,13 @@ def kv_workspace_bytes(model: Model, op: int, max_tokens: int) -> int:
     if r < 0:
         raise KVError(int(r), "kv_workspace_bytes")
     return int(r)
+
+
+def kv_workspace_residual(model: Model, op: int, max_tokens: int):
+    """(offset, bytes) of the fp32 residual stream inside a workspace sized for (op, max_tokens)."""
+    off, nbytes = C.c_int64(), C.c_int64()
+    _check(load().kv_workspace_residual(model.handle, op, max_tokens, C.byref(off), C.byref(nbytes)), "kv_workspace_residual")
+    return int(off.value), int(nbytes.value)
 
 
 def kv_check_device_status(workspace, stream=None) -> None:

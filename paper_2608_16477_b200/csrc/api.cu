@@ -183,14 +183,16 @@ struct PrefillWs {
   long long bytes;
 };
 
-PrefillWs carve_prefill(const kv_model_desc &d, void *base, int max_tokens, int block_size) {
+// The layout depends on the model and on max_tokens only (the block table is sized for one block per token), so
+// kv_workspace_bytes and kv_workspace_residual describe exactly what the operations carve.
+PrefillWs carve_prefill(const kv_model_desc &d, void *base, int max_tokens, int /*block_size*/) {
   Carver c(base);
   PrefillWs w;
   const long long t = max_tokens;
   const long long qkv_dim = (long long)(d.n_q_heads + 2 * d.n_kv_heads) * d.head_dim;
   w.status = c.take<DeviceStatus>(1);
   w.ids = c.take<int>(t);
-  w.table = c.take<int>((t + block_size - 1) / block_size + 1);
+  w.table = c.take<int>(t + 1);
   w.row_meta = c.take<int>(2 * t);
   w.rope = c.take<float2>(t * (d.head_dim / 2));
   w.x = c.take<float>(t * d.hidden);
@@ -212,12 +214,12 @@ struct DecodeWs {
   long long bytes;
 };
 
-DecodeWs carve_decode(const kv_model_desc &d, void *base, int max_ctx, int block_size) {
+DecodeWs carve_decode(const kv_model_desc &d, void *base, int max_ctx, int /*block_size*/) {
   Carver c(base);
   DecodeWs w;
   const long long qkv_dim = (long long)(d.n_q_heads + 2 * d.n_kv_heads) * d.head_dim;
   w.status = c.take<DeviceStatus>(1);
-  w.table = c.take<int>((max_ctx + block_size - 1) / block_size + 1);
+  w.table = c.take<int>(max_ctx + 1);
   w.rope = c.take<float2>(d.head_dim / 2);
   w.x = c.take<float>(d.hidden);
   w.h = c.take<float>(d.hidden);
@@ -313,6 +315,26 @@ int64_t kv_workspace_bytes(const kv_model *m, int32_t op, int32_t max_tokens) {
   if (m == nullptr || max_tokens <= 0) return KV_ERR_ARG;
   if (op == KV_OP_PREFILL) return carve_prefill(m->d, nullptr, max_tokens, 1).bytes;
   if (op == KV_OP_DECODE) return carve_decode(m->d, nullptr, max_tokens, 1).bytes;
+  return KV_ERR_ARG;
+}
+
+int32_t kv_workspace_residual(const kv_model *m, int32_t op, int32_t max_tokens, int64_t *offset_out,
+                              int64_t *bytes_out) {
+  if (m == nullptr || max_tokens <= 0 || offset_out == nullptr || bytes_out == nullptr) return KV_ERR_ARG;
+  // carve over a made-up base address (never dereferenced) to learn where the piece sits
+  char *fake = reinterpret_cast<char *>((uintptr_t)1 << 40);
+  if (op == KV_OP_PREFILL) {
+    const PrefillWs w = carve_prefill(m->d, fake, max_tokens, 1);
+    *offset_out = (int64_t)(reinterpret_cast<const char *>(w.x) - fake);
+    *bytes_out = (int64_t)max_tokens * m->d.hidden * 4;
+    return KV_OK;
+  }
+  if (op == KV_OP_DECODE) {
+    const DecodeWs w = carve_decode(m->d, fake, max_tokens, 1);
+    *offset_out = (int64_t)(reinterpret_cast<const char *>(w.x) - fake);
+    *bytes_out = (int64_t)m->d.hidden * 4;
+    return KV_OK;
+  }
   return KV_ERR_ARG;
 }
 

@@ -86,6 +86,73 @@ def test_32b_full_depth_properties(kv):
     assert rel <= exact_bound(s.n_layers), rel
 
 
+def test_32b_full_depth_single_layers_against_oracle(kv):
+    """Single layers of the 64-layer 32B-shaped model at the benchmark's prefix length, each against the oracle on that
+    layer's TRUE input.
+
+    The oracle cannot run 64 layers of this shape in test time, but it can run ONE layer of it.  A K/V-only prefill of
+    the first l + 1 layers leaves the input x_l of layer l in the workspace's residual stream and that layer's K/V in
+    the cache; the same prefill with logits leaves the layer's output x_{l+1}.  The oracle evaluates the layer on the
+    GPU's own x_l (all 4,096 rows), so nothing accumulates and the bounds are those of a first layer:
+      * K/V of layers 1, 15, 31, 47 and 63 within exact_bound(0) of the oracle (3.5e-3; the floor of two-byte storage is 2.35e-3);
+      * the update x_{l+1} - x_l of the LAST layer (attention, O projection, SwiGLU FFN at K = 8,192 and 25,600 in the
+        benchmark's instantiations) within 1.5 x the distance the oracle's own bf16-storage evaluation has from its exact
+        one, and close to that bf16-storage evaluation."""
+    import torch
+    s = synth.SHAPES["32b"]
+    s = synth.ModelShape(**{**s.__dict__, "vocab": 4096})
+    prefix = 4096
+    bs = s.block_size
+    gen = torch.Generator(device="cuda").manual_seed(11)
+
+    def mat(r, c):
+        return torch.empty(r, c, dtype=torch.bfloat16, device="cuda").normal_(0.0, s.init_std, generator=gen)
+    ones = lambda: torch.ones(s.hidden, dtype=torch.bfloat16, device="cuda")
+    W = [{"attn_norm": ones(), "ffn_norm": ones(), "w_qkv": mat(s.qkv_dim, s.hidden), "w_o": mat(s.hidden, s.q_dim),
+          "w_gate_up": mat(2 * s.ffn, s.hidden), "w_down": mat(s.hidden, s.ffn)} for _ in range(s.n_layers)]
+    head = {"embed": mat(s.vocab, s.hidden), "lm_head": mat(s.vocab, s.hidden), "final_norm": ones()}
+    ids = synth.token_ids(s, 11, prefix)
+    table = synth.block_permutation(12, 512)[: prefix // bs]
+    pos = np.arange(prefix)
+    logits = torch.empty(s.vocab, dtype=torch.float32, device="cuda")
+
+    def residual(model, ws):
+        off, nbytes = kv.kv_workspace_residual(model, kv.KV_OP_PREFILL, prefix)
+        return ws[off:off + nbytes].view(torch.float32).view(prefix, s.hidden).cpu().numpy().astype(np.float64)
+
+    for l, whole_layer in ((1, False), (15, False), (31, False), (47, False), (63, True)):
+        sub = s.with_layers(l + 1)
+        model = kv.Model(sub, head, lambda i: W[i])             # shares the device tensors, no copies
+        cache = kv.PagedCache(sub, 512, fill=0)
+        ws = kv.kv_prefill_prefix(model, cache, ids, table)      # K/V only: the last layer stops after its K/V
+        kv.kv_check_device_status(ws)
+        x_in = residual(model, ws)
+        img = cache.data[l].cpu().numpy().view(np.uint16).reshape(1, 2, 512, bs, s.n_kv_heads, s.head_dim)
+        Kg, Vg = O.read_kv(img, table, prefix)
+        w_host = {k: v.float().cpu().numpy() for k, v in W[l].items()}
+        _, Kref, Vref = O.layer_forward(s, w_host, x_in, pos, mm_dtype=np.float32, skip_after_kv=True)
+        for nm, got, ref in (("K", Kg[0], Kref), ("V", Vg[0], Vref)):
+            st = error_stats(got, ref)
+            print(f"32b layer {l} {nm} on its true input:", st)
+            assert st["rel_l2"] <= exact_bound(0) and elementwise_ok(got, ref, exact_bound(0)), (l, nm, st)
+        if not whole_layer:
+            continue
+        ws = kv.kv_prefill_prefix(model, cache, ids, table, logits_out=logits)     # now the last layer runs to its end
+        kv.kv_check_device_status(ws)
+        x_out = residual(model, ws)
+        xe, _, _ = O.layer_forward(s, w_host, x_in, pos, mm_dtype=np.float32)
+        xb, _, _ = O.layer_forward(s, w_host, x_in, pos, mm_dtype=np.float32, act_bf16=True)
+        u_ref = xe - x_in
+        norm = float(np.sqrt(np.sum(u_ref ** 2)))
+        floor = float(np.sqrt(np.sum((xb - xe) ** 2))) / norm
+        vs_exact = float(np.sqrt(np.sum((x_out - xe) ** 2))) / norm
+        vs_storage = float(np.sqrt(np.sum((x_out - xb) ** 2))) / norm
+        print(f"32b layer {l} update x_out - x_in: oracle floor {floor:.4e}, GPU vs exact {vs_exact:.4e}, "
+              f"GPU vs bf16-storage oracle {vs_storage:.4e}, |update| / |x| {norm / np.sqrt(np.sum(x_in ** 2)):.3e}")
+        assert vs_exact <= 1.5 * floor, (vs_exact, floor)
+        assert vs_storage <= floor, (vs_storage, floor)
+
+
 def test_32b_full_size_pack_unpack_sampled(kv):
     import torch
     s = synth.SHAPES["32b"]
