@@ -391,6 +391,9 @@ def run_ours(args):
             return timed(fn, reps) / (reps * n_sets), "direct launches"
     pack_ms, pack_how = graph_time(pack_all)
     unpack_ms, _ = graph_time(unpack_all)
+    # the same launches issued directly (no graph): what the gaps between short launches cost by themselves
+    pack_direct_ms = timed(pack_all, 10) / (10 * n_sets)
+    unpack_direct_ms = timed(unpack_all, 10) / (10 * n_sets)
 
     # the decode step timed alone as well (direct launches), before the prefill pulls the clocks down
     merged0 = kv.kv_unpack_assemble(tgt, wire, logical, dst_ids, tgt_prefix, n, epoch=1, expected_epoch=1)
@@ -505,10 +508,13 @@ def run_ours(args):
         "pack": {"gbs": 2 * payload / (pack_ms * 1e-3) / 1e9, "frac_of_hbm": 2 * payload / (pack_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
                  "us": pack_ms * 1e3, "payload_bytes": payload,
                  "timing": f"{pack_how} of {n_sets} launches over disjoint block sets",
+                 "direct_launch_us": pack_direct_ms * 1e3,
                  "in_step_us": per_step["pack"][0] * 1e3,
-                 "frac_in_step": 2 * payload / (per_step["pack"][0] * 1e-3) / 1e9 / pk["hbm_gbs"]},
+                 "frac_in_step": 2 * payload / (per_step["pack"][0] * 1e-3) / 1e9 / pk["hbm_gbs"],
+                 "in_step_note": "CUDA events around the one launch, right behind the power-capped prefill"},
         "unpack": {"gbs": 2 * payload / (unpack_ms * 1e-3) / 1e9,
                    "frac_of_hbm": 2 * payload / (unpack_ms * 1e-3) / 1e9 / pk["hbm_gbs"], "us": unpack_ms * 1e3,
+                   "direct_launch_us": unpack_direct_ms * 1e3,
                    "in_step_us": per_step["unpack"][0] * 1e3,
                    "frac_in_step": 2 * payload / (per_step["unpack"][0] * 1e-3) / 1e9 / pk["hbm_gbs"]},
         "decode_step_ms": decode_ms,

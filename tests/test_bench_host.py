@@ -29,3 +29,25 @@ def test_peaks_have_every_key():
     p = bench.peaks()
     assert p["source"] in ("measured", "fallback")
     assert p["hbm_gbs"] > 0 and p["bf16_tflops"] >= p["bf16_tflops_sustained"] > 0
+
+
+def test_both_arms_describe_the_same_workload_and_sample():
+    """The GPU arm and the reference arm print the same `config` and size the oracle's bounded sample with the same
+    function: the whole 4,096-token prefix for a default run, half of it when 25 runs were asked for (so that the
+    reference arm ends within a few minutes), a quarter beyond 40 runs."""
+    a = bench.workload_config("32b-4k", world=1)
+    assert a["workload"] == "32b-4k" and a["prefix_tokens"] == 4096 and a["suffix_tokens"] == 512 and a["layers"] == 64
+    assert a == bench.workload_config("32b-4k", world=1)
+    assert bench.workload_config("32b-4k", world=8)["parallelism"] == "replicas x8"
+    assert bench.oracle_sample_tokens(4096, 4096, 3, 3) == 4096
+    assert bench.oracle_sample_tokens(4096, 4096, 20, 5) == 2048
+    assert bench.oracle_sample_tokens(4096, 4096, 50, 5) == 1024
+    assert bench.oracle_sample_tokens(128, 4096, 3, 3) == 128
+    assert bench.oracle_sample_tokens(4096, 1000, 3, 3) == 1000
+
+
+def test_tensor_pipe_ceiling_model():
+    # 148 SMs x 8,192 bf16 flop per clock per SM (one 128 x 128 x 16 MMA per 64 cycles)
+    assert 2 * 128 * 128 * 16 // 64 == bench.BF16_FLOP_PER_CLK_PER_SM
+    assert bench.hw_tensor_peak_tflops(1965.0) == pytest.approx(2382.6, abs=0.5)
+    assert bench.hw_tensor_peak_tflops(1282.0) == pytest.approx(1554.3, abs=0.5)
