@@ -98,16 +98,24 @@ def prefill_flops(shape, n_tokens, with_logits=False):
 
 
 # ------------------------------------------------------------------------------------------ reference arm
-def oracle_sample(shape, n_tokens, seed=0):
-    """Bounded sample of the workload for the CPU oracle: ONE decoder layer over the first n_tokens prefix tokens."""
+def oracle_sample(shape, n_tokens, prefix=None, seed=0):
+    """Bounded sample of the workload for the CPU oracle: ONE decoder layer over n_tokens rows of the prefix.  When the
+    sample is shorter than the prefix it is the MIDDLE of it (rows (prefix - n) / 2 ... attending to the cached rows
+    before them), so that a row sees as many keys on average as a row of the whole prefix does and attention keeps
+    its true share of the work."""
     from oracle import kv_oracle as O
+    prefix = n_tokens if prefix is None else prefix
+    start = (prefix - n_tokens) // 2
     w = synth.layer_weights(shape, seed, 0)
-    x = (np.random.default_rng(seed).standard_normal((n_tokens, shape.hidden)) * shape.init_std)
-    pos = np.arange(n_tokens)
+    rng = np.random.default_rng(seed)
+    x = rng.standard_normal((n_tokens, shape.hidden)) * shape.init_std
+    k_past = rng.standard_normal((start, shape.n_kv_heads, shape.head_dim)) if start else None
+    v_past = rng.standard_normal((start, shape.n_kv_heads, shape.head_dim)) if start else None
+    pos = np.arange(start, start + n_tokens)
 
     def run():
         t0 = time.perf_counter()
-        O.layer_forward(shape, w, x, pos)
+        O.layer_forward(shape, w, x, pos, k_past=k_past, v_past=v_past)
         return time.perf_counter() - t0
     return run
 
@@ -151,14 +159,17 @@ def oracle_sample_tokens(prefix, cap, steps, warmup):
 
 
 def oracle_sample_text(shape, prefix, sample_tokens):
-    part = "the whole prefix" if sample_tokens == prefix else f"the first {sample_tokens} of {prefix} prefix tokens"
+    part = ("the whole prefix" if sample_tokens == prefix else
+            f"the middle {sample_tokens} of {prefix} prefix tokens (rows {(prefix - sample_tokens) // 2} to "
+            f"{(prefix + sample_tokens) // 2 - 1}, attending to the cached rows before them: the same mean number of "
+            f"keys per row as over the whole prefix)")
     return (f"one decoder layer (1 of {shape.n_layers}) of the fp64 numpy oracle over {part}; tokens/s extrapolated "
             f"to {shape.n_layers} layers")
 
 
 def cpu_baseline(shape, prefix, sample_tokens, repeats=3, suffix_blocks=0):
     """The oracle as it stands on the host cores: best of `repeats` runs of the bounded sample."""
-    run = oracle_sample(shape, sample_tokens)
+    run = oracle_sample(shape, sample_tokens, prefix)
     times = [run() for _ in range(repeats)]
     secs = min(times)
     value = sample_tokens / (secs * shape.n_layers)
@@ -179,7 +190,7 @@ def run_reference(args):
     shape = synth.SHAPES[shape_name]
     warmup = max(args.ref_warmup, args.warmup if args.warmup_given else 0)
     sample_tokens = oracle_sample_tokens(prefix, args.ref_tokens, args.steps, warmup)
-    run = oracle_sample(shape, sample_tokens)
+    run = oracle_sample(shape, sample_tokens, prefix)
     for _ in range(warmup):
         run()
     times = [run() for _ in range(args.steps)]
