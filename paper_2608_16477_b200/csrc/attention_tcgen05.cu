@@ -131,10 +131,8 @@ __device__ __forceinline__ float ex2_approx(float x) {
 // below the bf16 rounding the probabilities get anyway), then n is added into the exponent field.  Arguments are
 // clamped at -126, so masked scores (minus infinity) come out as 2^-126 instead of 0: eight orders of magnitude
 // below anything a bf16 sum or product can notice.
-#ifndef KV_ATTN_POLY_PAIRS
-#define KV_ATTN_POLY_PAIRS 4     // pairs per 16-pair chunk whose exponentials take this path (4: a quarter of all)
-#endif
-constexpr int kPolyPairs = KV_ATTN_POLY_PAIRS;
+constexpr int kPolyPairs = 4;     // pairs per 16-pair chunk whose exponentials take this path (a quarter of all:
+                                  // measured best among 0, 2, 4, 6, 8 and 16)
 __device__ __forceinline__ void exp2_pair_fma(uint64_t x2, float &p0, float &p1) {
   float x0, x1;
   unpk2(x2, x0, x1);

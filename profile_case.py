@@ -1,8 +1,9 @@
 """Runs ONE kernel of the hot path a few times at the benchmark's shapes, for profiler captures.
 
   python profile_case.py gemm_gate_up [--tokens 4096] [--iters 3]
-  cases: gemm_qkv, gemm_o, gemm_gate_up, gemm_down, attention, pack, unpack, pack_batched, unpack_batched, decode_gemv,
-         decode_gemv_o, decode_attention, prefill_layer
+  cases: gemm_qkv, gemm_o, gemm_gate_up, gemm_down, attention, rmsnorm, pack, unpack, pack_batched, unpack_batched,
+         decode_gemv (gate/up), decode_gemv_o, decode_gemv_down, decode_gemv_qkv, decode_gemv_lm_head, decode_attention,
+         prefill_layer
 
 Inputs are synthetic and larger than L2 where the kernel is bandwidth-bound; a few GB at most are held on
 the device so a multi-pass capture stays short.  Prints the CUDA-event time per launch.
@@ -107,18 +108,35 @@ def main():
             else:
                 kv.kv_unpack_blocks_batched(cache, offs, perms[i], wires[i])
         work, unit = 2.0 * int(offs[-1]) * block_bytes / 1e9, "GB/s"
-    elif a.case == "decode_gemv_o":
-        # the O projection of one decode step (5120 x 8192, 84 MB: a SHORT launch), residual-add epilogue, rotating over
-        # 6 weight copies (> L2)
-        ws = [rnd(s.hidden, s.q_dim, std=0.02) for _ in range(6)]
-        x = torch.randn(s.q_dim, device=dev)
-        y = torch.zeros(s.hidden, device=dev)
+    elif a.case in ("decode_gemv_o", "decode_gemv_down", "decode_gemv_qkv", "decode_gemv_lm_head"):
+        # the other products of one decode step, each as its own (SHORT) launch, rotating over enough weight copies to
+        # exceed L2: O projection 5120 x 8192 (84 MB, residual add), down projection 5120 x 25600 (262 MB, residual add),
+        # a QKV-sized product 10240 x 5120 (105 MB, norm folded in), the LM head 151936 x 5120 (1.56 GB, norm folded in)
+        rows, k, mode, norm = {"decode_gemv_o": (s.hidden, s.q_dim, 1, False), "decode_gemv_down": (s.hidden, s.ffn, 1, False),
+                               "decode_gemv_qkv": (s.qkv_dim, s.hidden, 0, True),
+                               "decode_gemv_lm_head": (s.vocab, s.hidden, 0, True)}[a.case]
+        copies = max(2, int(400e6 // (rows * k * 2)) + 1)
+        ws = [rnd(rows, k, std=0.02) for _ in range(copies)]
+        x = torch.randn(k, device=dev)
+        gain = torch.ones(k, dtype=torch.bfloat16, device=dev) if norm else None
+        y = torch.zeros(rows, device=dev)
         state = {"i": 0}
 
         def run():
             state["i"] += 1
-            kv.kv_op_gemv(ws[state["i"] % 6], x, 1, y)
+            kv.kv_op_gemv(ws[state["i"] % copies], x, mode, y, gain=gain, eps=1e-6)
         work, unit = ws[0].numel() * 2 / 1e9, "GB/s"
+    elif a.case == "rmsnorm":
+        # one normalisation pass of the prefill: tokens x hidden fp32 -> bf16, rotating over four inputs (> L2)
+        xs = [torch.randn(t, s.hidden, device=dev) for _ in range(4)]
+        gain = torch.ones(s.hidden, dtype=torch.bfloat16, device=dev)
+        outs = [torch.empty(t, s.hidden, dtype=torch.bfloat16, device=dev) for _ in range(4)]
+        state = {"i": 0}
+
+        def run():
+            state["i"] += 1
+            kv.kv_op_rmsnorm(xs[state["i"] % 4], gain, 1e-6, outs[state["i"] % 4])
+        work, unit = t * s.hidden * 6 / 1e9, "GB/s"
     elif a.case == "decode_gemv":
         # the gate/up product of one decode step (524 MB of weights), rotating over 4 weight copies (> L2)
         ws = [rnd(2 * s.ffn, s.hidden, std=0.02) for _ in range(4)]

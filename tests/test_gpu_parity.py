@@ -84,6 +84,43 @@ def test_pack_ragged_and_empty(kv, torch):
     assert np.array_equal(dst.as_logical_numpy(), want)
 
 
+def test_pack_unpack_beyond_one_parameter_block(kv, torch):
+    """More blocks (9,001) than one launch's parameter block carries (7,680) in a single request, and more requests
+    (70) than it has records for (64) in a batched call: the lists continue in further launches, a request may
+    straddle two of them, and every page still lands where the oracle puts it."""
+    s = synth.ModelShape("odd", n_layers=2, hidden=64, n_q_heads=1, n_kv_heads=1, head_dim=32, ffn=64, vocab=16,
+                         block_size=1)
+    nb = 9100
+    rng = np.random.default_rng(13)
+    img = rng.integers(0, 65536, (2, 2, nb, 1, 1, 32)).astype(np.uint16)
+    src = kv.PagedCache(s, nb)
+    src.data.copy_(_bits_to_torch(torch, img.reshape(2, 2, nb, 32)))
+    ids = synth.block_permutation(14, nb)[:9001]
+    for layout in (0, 1):
+        wire = torch.zeros(9001 * 2 * 2 * 32, dtype=torch.int16, device="cuda")
+        kv.kv_pack_blocks(src, ids, wire, wire_layout=layout)
+        want = O.pack_blocks(img, ids)
+        if layout == 1:
+            want = want.transpose(1, 2, 0, 3)
+        assert np.array_equal(wire.cpu().numpy().view(np.uint16), want.reshape(-1)), layout
+    # 70 requests of 1..9 blocks each through the batched calls
+    counts = [1 + (i * 7) % 9 for i in range(70)]
+    offs = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+    rid = synth.block_permutation(15, nb)[: offs[-1]]
+    wires = [torch.zeros(c * 2 * 2 * 32, dtype=torch.int16, device="cuda") for c in counts]
+    kv.kv_pack_blocks_batched(src, offs, rid, wires)
+    for r, c in enumerate(counts):
+        want = O.pack_blocks(img, rid[offs[r]:offs[r + 1]])
+        assert np.array_equal(wires[r].cpu().numpy().view(np.uint16), want.reshape(-1)), r
+    dst = kv.PagedCache(s, nb, fill=0)
+    did = synth.block_permutation(16, nb)[: offs[-1]]
+    kv.kv_unpack_blocks_batched(dst, offs, did, wires)
+    want_img = np.zeros_like(img)
+    want_img[:, :, did] = img[:, :, rid]
+    assert np.array_equal(dst.as_logical_numpy(), want_img)
+    kv.kv_check_copy_status()
+
+
 def test_pack_unpack_batched_pattern_32b_pages(kv, torch):
     """32 KiB pages, 64 layers: a scaled-down form of the 16-request stress workload whose content is the
     counter-based pattern, checked page by page against the host generator."""
