@@ -131,7 +131,9 @@ def oracle_reference_bf16_storage(shape, seed, ids, k, mm_dtype=np.float64):
     L, _, hkv, d = Kp.shape
     Kc = np.zeros((L, n + 1, hkv, d)); Vc = np.zeros((L, n + 1, hkv, d))
     Kc[:, :k], Vc[:, :k] = Kp, Vp
-    all_layers = [synth.layer_weights(shape, seed, l) for l in range(shape.n_layers)]
+    # held as fp64 once: the incremental step would otherwise convert every matrix on every call
+    all_layers = [{k: np.asarray(v, dtype=np.float64) for k, v in synth.layer_weights(shape, seed, l).items()}
+                  for l in range(shape.n_layers)]
     logits = None
     for pos in range(k, n + 1):
         kn, vn, logits = O.decode_step(shape, head, lambda l: all_layers[l], ids[pos], pos, Kc, Vc)
