@@ -97,6 +97,28 @@ def prefill_flops(shape, n_tokens, with_logits=False):
     return L * qkv + full_layers * (rest + attn)
 
 
+def step_work(shape, prefix, suffix):
+    """Algorithmic work of one bench step per kernel class: (amount, unit) with flops for the tensor-bound classes
+    and bytes (read + written) for the HBM-bound ones.  K/V-only prefill: the last layer stops after its QKV projection."""
+    d, qd, kvd, f, L = shape.hidden, shape.q_dim, shape.kv_dim, shape.ffn, shape.n_layers
+    n = prefix
+    n_ctx = prefix + suffix + 1
+    page_payload = -(-suffix // shape.block_size) * L * 2 * synth.kv_page_bytes(shape)
+    return {
+        "gemm_qkv": (L * 2.0 * n * d * (qd + 2 * kvd), "flop"),
+        "attention": ((L - 1) * 2.0 * shape.n_q_heads * shape.head_dim * n * (n + 1), "flop"),
+        "gemm_o": ((L - 1) * 2.0 * n * qd * d, "flop"),
+        "gemm_gate_up": ((L - 1) * 2.0 * n * d * 2 * f, "flop"),
+        "gemm_down": ((L - 1) * 2.0 * n * f * d, "flop"),
+        "rmsnorm": ((2 * L - 1) * n * d * 6.0, "byte"),
+        "pack": (2.0 * page_payload, "byte"),
+        "unpack": (2.0 * page_payload, "byte"),
+        "decode_gemv": (L * 2.0 * (d * (qd + 2 * kvd) + qd * d + 3 * d * f), "byte"),
+        "decode_attention": (L * 2.0 * n_ctx * kvd * 2, "byte"),
+        "lm_head": (2.0 * shape.vocab * d, "byte"),
+    }
+
+
 # ------------------------------------------------------------------------------------------ reference arm
 def oracle_sample(shape, n_tokens, prefix=None, seed=0):
     """Bounded sample of the workload for the CPU oracle: ONE decoder layer over n_tokens rows of the prefix.  When the
@@ -543,6 +565,21 @@ def run_ours(args):
         "t0_analog_ms": per_step["unpack"][0] + decode_ms,
         "breakdown_ms_per_step": {k: round(v[0], 4) for k, v in per_step.items()},
     }
+    # every kernel class of the step against the measured peak that bounds it (the library matmul's sustained rate
+    # for the tensor-bound classes, the copy bandwidth for the HBM-bound ones), from the event times above
+    if not args.layers:
+        table = {}
+        for kind, (amount, unit) in step_work(shape, prefix, suffix).items():
+            ms = per_step[kind][0]
+            if ms <= 0:
+                continue
+            if unit == "flop":
+                rate = amount / (ms * 1e-3) / 1e12
+                table[kind] = {"ms": round(ms, 3), "tflops": round(rate, 1), "frac_of_sustained_peak": round(rate / pk["bf16_tflops_sustained"], 3)}
+            else:
+                rate = amount / (ms * 1e-3) / 1e9
+                table[kind] = {"ms": round(ms, 4), "gbs": round(rate, 1), "frac_of_hbm": round(rate / pk["hbm_gbs"], 3)}
+        line["kernel_rooflines_in_step"] = table
     if sweep:
         line["sweep"] = sweep
     # Algorithm 1 fed with the rates measured above (Section 4.2): prefill rate r_p, decode rate r_d of the

@@ -51,3 +51,13 @@ def test_tensor_pipe_ceiling_model():
     assert 2 * 128 * 128 * 16 // 64 == bench.BF16_FLOP_PER_CLK_PER_SM
     assert bench.hw_tensor_peak_tflops(1965.0) == pytest.approx(2382.6, abs=0.5)
     assert bench.hw_tensor_peak_tflops(1282.0) == pytest.approx(1554.3, abs=0.5)
+
+
+def test_step_work_adds_up():
+    s = synth.SHAPES["32b"]
+    w = bench.step_work(s, 4096, 512)
+    flops = sum(a for a, u in w.values() if u == "flop")
+    assert flops == pytest.approx(bench.prefill_flops(s, 4096))            # the classes cover the whole prefill
+    assert w["pack"][0] == 2 * 32 * 64 * 2 * 32768 == w["unpack"][0]       # 128 MiB read + 128 MiB written
+    assert w["decode_gemv"][0] / 1e9 == pytest.approx(62.41, abs=0.01)     # every layer's weights once
+    assert w["rmsnorm"][0] == 127 * 4096 * 5120 * 6
