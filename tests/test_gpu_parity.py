@@ -299,6 +299,29 @@ def test_attention_prefill_kernel_over_cached_prefix(kv, torch, pos0, t, hq, hkv
     assert st["max_abs"] <= MAX_ABS and st["rel_l2"] <= REL_L2, st
 
 
+@pytest.mark.parametrize("scale", [4.0, 12.0])
+def test_attention_prefill_kernel_wide_score_range(kv, torch, scale):
+    """Scores with a standard deviation of 16 and 144 instead of 1: running maxima that jump by far more than the lazy
+    rescaling threshold, exponents far below the clamp of the FMA-pipe exponential (2^-126), rows dominated by a single
+    key.  Every exponential path (special-function unit, polynomial, masked) must agree with the oracle."""
+    t, hq, hkv, d = 700, 4, 2, 128
+    rng = np.random.default_rng(int(scale) + 40)
+    qkv = rng.standard_normal((t, (hq + 2 * hkv) * d), dtype=np.float32)
+    qkv[:, : (hq + hkv) * d] *= np.float32(scale)                    # queries and keys
+    qkv = synth.bf16_round_f32(qkv)
+    q = qkv[:, : hq * d].reshape(t, hq, d)
+    k = qkv[:, hq * d: (hq + hkv) * d].reshape(t, hkv, d)
+    v = qkv[:, (hq + hkv) * d:].reshape(t, hkv, d)
+    want = O.attention(q, k, v)
+    out = torch.empty(t, hq * d, dtype=torch.bfloat16, device="cuda")
+    status = torch.zeros(64, dtype=torch.int32, device="cuda")
+    kv.kv_op_attention_prefill(torch.from_numpy(qkv).cuda().to(torch.bfloat16), hq, hkv, d, out, status=status)
+    got = out.float().cpu().numpy().reshape(t, hq, d)
+    assert int(status[0]) == 0 and np.all(np.isfinite(got))
+    st = error_stats(got, want)
+    assert st["max_abs"] <= MAX_ABS and st["rel_l2"] <= REL_L2, st
+
+
 def test_attention_prefill_long_context_sampled_rows(kv, torch):
     """8,192 tokens (64 key tiles for the last row tile, 256 work items on 148 SMs): three windows of query rows are
     checked against the oracle, which scores each window against the keys up to its last row."""
