@@ -401,6 +401,23 @@ def test_scenario_tiny(kv, name, n_suffix):
     assert st["rel_l2"] <= REL_L2, st
 
 
+def test_scenario_odd_query_group(kv):
+    """Three query heads per KV head (an odd group: the prefill attention pairs the third head with itself) and one
+    query head per KV head, through the whole path against the oracle."""
+    for hq, hkv in ((6, 2), (2, 2)):
+        s = synth.ModelShape(f"odd{hq}", n_layers=2, hidden=192, n_q_heads=hq, n_kv_heads=hkv, head_dim=64, ffn=384,
+                             vocab=512, sharp=True)
+        ids = synth.token_ids(s, 0, 150)
+        Kref, Vref, logits_ref = oracle_reference(s, 0, ids)
+        res = run_gpu_scenario(kv, s, 0, ids, 112, 149)
+        assert np.array_equal(res["merged"], res["expected_merged"])
+        for name, got, ref in (("K", res["K"], Kref), ("V", res["V"], Vref), ("logits", res["logits"], logits_ref)):
+            st = error_stats(got, ref)
+            assert st["rel_l2"] <= REL_L2 and st["scaled_ok"], (hq, name, st)
+        _, _, lp = oracle_reference(s, 0, ids[:112])
+        assert error_stats(res["prefill_logits"], lp)["rel_l2"] <= REL_L2
+
+
 def test_scenario_tiny_block_major_layer_major_wire(kv):
     s = synth.SHAPES["tiny-sharp"]
     ids = synth.token_ids(s, 0, 161)
