@@ -745,6 +745,98 @@ def run_batched_prefill(args):
     return 0
 
 
+def run_chunk_interleave(args):
+    """Contention-aware migration (Section 4.5): the target keeps serving a resident request while it rebuilds a
+    migrating request's 4,096-token prefix in chunks, one resident decode step after every chunk, on one stream.
+    Reports, for 256-token chunks (the chunk size of Section 6.3) and 1,024-token chunks, what the resident request
+    sees (time between its tokens while the migration runs, against its undisturbed decode step) and what the
+    migration pays (chunked and interleaved rebuild against one uninterrupted prefill call), 32B shape."""
+    import torch
+    import paper_2608_16477_b200 as kv
+    kv.load()
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    shape = synth.SHAPES["32b"]
+    prefix, resident_ctx, chunk_sizes = 4096, 2048, (256, 1024)
+    bs = shape.block_size
+    max_steps = prefix // min(chunk_sizes)
+    res_blocks = (resident_ctx + max_steps) // bs + 1
+    mig_blocks = prefix // bs
+    model, _ = build_model(kv, torch, shape)
+    cache = kv.PagedCache(shape, res_blocks + mig_blocks + 8)
+    kv.kv_fill_pattern(cache.data, cache.data.numel() * 2, seed=5)
+    cache.data.bitwise_and_(0x3FFF)                    # finite bf16 content standing in for the resident request's K/V
+    perm = synth.block_permutation(1, res_blocks + mig_blocks + 8)
+    res_table, mig_table = perm[:res_blocks], perm[res_blocks:res_blocks + mig_blocks]
+    res_ids = synth.token_ids(shape, 0, resident_ctx + max_steps + 1)
+    mig_ids = synth.token_ids(shape, 1, prefix)
+    logits = torch.empty(shape.vocab, dtype=torch.float32, device="cuda")
+    ws_d = model.workspace(kv.KV_OP_DECODE, resident_ctx + max_steps + 1)
+    ws_p = model.workspace(kv.KV_OP_PREFILL, prefix)
+    stream = torch.cuda.current_stream()
+
+    def decode(i):
+        pos = resident_ctx + i
+        kv.kv_decode_step(model, cache, int(res_ids[pos]), pos, res_table[: pos // bs + 1], logits, workspace=ws_d)
+
+    def prefill_chunk(c, chunk):
+        kv.kv_prefill_prefix(model, cache, mig_ids[c * chunk:(c + 1) * chunk], mig_table[: (c + 1) * chunk // bs],
+                             pos0=c * chunk, workspace=ws_p)
+
+    def measure(fn):
+        for _ in range(max(args.warmup, 3)):
+            fn()
+        best = None
+        for _ in range(args.steps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record(stream)
+            fn()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1)
+            best = ms if best is None else min(best, ms)
+        return best
+
+    def decode_alone():
+        for i in range(max_steps):
+            decode(i)
+
+    def chunked(chunk, with_decode):
+        def run():
+            for c in range(prefix // chunk):
+                prefill_chunk(c, chunk)
+                if with_decode:
+                    decode(c)
+        return run
+
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    l0 = kv.kv_launch_count()
+    itl_alone = measure(decode_alone) / max_steps
+    one_call = measure(lambda: kv.kv_prefill_prefix(model, cache, mig_ids, mig_table, workspace=ws_p))
+    per_chunk = {}
+    for chunk in chunk_sizes:
+        alone, busy = measure(chunked(chunk, False)), measure(chunked(chunk, True))
+        itl = busy / (prefix // chunk)
+        per_chunk[str(chunk)] = {"rebuild_ms": alone, "rebuild_ms_with_resident_decode": busy,
+                                 "rebuild_vs_one_call": alone / one_call, "resident_ms_between_tokens": itl,
+                                 "resident_slowdown": itl / itl_alone}
+    launches = kv.kv_launch_count() - l0
+    clocks = sampler.stop()
+    kv.kv_check_device_status(ws_p)
+    head = per_chunk[str(chunk_sizes[0])]
+    line = {"metric": METRIC, "value": prefix / (head["rebuild_ms_with_resident_decode"] * 1e-3), "unit": UNIT, "n_gpus": 1,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": head["rebuild_ms_with_resident_decode"],
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "chunk-interleave", "shape": "32b", "prefix_tokens": prefix,
+                       "chunk_tokens": list(chunk_sizes), "resident_context": resident_ctx,
+                       "l2": "weights (62 GB per pass) larger than L2"},
+            "rebuild_ms_one_call": one_call, "resident_ms_between_tokens_alone": itl_alone, "chunks": per_chunk,
+            "clocks": clocks, "gpu_launches": int(launches)}
+    print(json.dumps(line))
+    return 0
+
+
 def run_pack_stress(args):
     import torch
     import paper_2608_16477_b200 as kv
@@ -806,7 +898,7 @@ def main():
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="32b-4k", choices=sorted(WORKLOADS) + ["pack-stress", "stream-overlap", "batched-prefill"])
+    ap.add_argument("--workload", default="32b-4k", choices=sorted(WORKLOADS) + ["pack-stress", "stream-overlap", "batched-prefill", "chunk-interleave"])
     ap.add_argument("--layers", type=int, default=0, help="debug: reduced depth (invalid as a bench number)")
     ap.add_argument("--ref-tokens", type=int, default=4096, help="prefix tokens in the oracle's bounded sample")
     ap.add_argument("--ref-warmup", type=int, default=0)
@@ -821,6 +913,8 @@ def main():
         return run_stream_overlap(args)
     if args.workload == "batched-prefill" and args.impl != "reference":
         return run_batched_prefill(args)
+    if args.workload == "chunk-interleave" and args.impl != "reference":
+        return run_chunk_interleave(args)
     if args.impl == "reference":
         return run_reference(args)
     return run_ours(args)

@@ -79,6 +79,43 @@ def test_chunked_prefill_against_oracle_tiny(kv, torch, name, chunks):
     assert not img[:, :, np.setdiff1d(np.arange(64), table)].any()
 
 
+@pytest.mark.parametrize("name", ["tiny", "tiny-sharp"])
+def test_chunked_prefill_interleaved_with_resident_decode(kv, torch, name):
+    """Section 4.5's schedule on one stream: a migrating request's prefix is rebuilt in chunks while a resident request
+    on the same model and the same block pool decodes one token after every chunk.  Both are checked against the
+    oracle: the resident request's logits at every step, the migrating request's K/V and first resumed token."""
+    s, head, lw, model = _tiny_model(kv, name, 7)
+    chunks = (48, 32, 16, 64)
+    n_mig, n_res = sum(chunks), 80
+    mig_ids = synth.token_ids(s, 8, n_mig + 1)
+    res_ids = synth.token_ids(s, 9, n_res + len(chunks) + 1)
+    Km, Vm, lm = O.forward_full(s, head, lambda l: lw[l], mig_ids)
+    perm = synth.block_permutation(10, 64)
+    res_table, mig_table = perm[:8], perm[8:8 + n_mig // 16 + 1]
+    cache = kv.PagedCache(s, 64, fill=0)
+    logits = torch.empty(s.vocab, dtype=torch.float32, device="cuda")
+    kv.kv_prefill_prefix(model, cache, res_ids[:n_res], res_table[: n_res // 16])
+    p0 = 0
+    for i, c in enumerate(chunks):
+        ws = kv.kv_prefill_prefix(model, cache, mig_ids[p0:p0 + c], mig_table[: (p0 + c) // 16], pos0=p0)
+        kv.kv_check_device_status(ws)
+        p0 += c
+        pos = n_res + i
+        kv.kv_decode_step(model, cache, int(res_ids[pos]), pos, res_table[: pos // 16 + 1], logits)
+        _, _, lref = O.forward_full(s, head, lambda l: lw[l], res_ids[: pos + 1])
+        st = error_stats(logits.cpu().numpy(), lref)
+        assert st["rel_l2"] <= STATED_REL_L2, ("resident", i, st)
+    Kg, Vg = _kv_of(cache, mig_table, n_mig)
+    _check_kv(s, Kg, Vg, Km[:, :n_mig], Vm[:, :n_mig], name == "tiny", "interleaved")
+    kv.kv_decode_step(model, cache, int(mig_ids[n_mig]), n_mig, mig_table, logits)
+    st = error_stats(logits.cpu().numpy(), lm)
+    assert st["rel_l2"] <= STATED_REL_L2, ("migrated", st)
+    # the two requests' pages are disjoint and nothing else was written
+    img = cache.as_logical_numpy()
+    used = np.concatenate([res_table[: (n_res + len(chunks)) // 16 + 1], mig_table])
+    assert not img[:, :, np.setdiff1d(np.arange(64), used)].any()
+
+
 @pytest.fixture(scope="module")
 def wide(kv):
     """A 32B-shaped two-layer model and the oracle's exact forward over 1,000 tokens (shared by the wide cases)."""
