@@ -299,7 +299,7 @@ attention_prefill_tc_kernel(const __grid_constant__ CUtensorMap tma_qkv, int n_t
     // sits on a third.
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
     {
-      // every lane waits, and the verdict is made uniform so that the warp stays converged for elect.sync
+      // every lane waits, and the outcome is made uniform so that the warp stays converged for elect.sync
       auto wwait = [&](uint32_t b_, uint32_t parity, volatile int *af, DeviceStatus *st_, int tag) {
         return __all_sync(0xffffffffu, tc::mbar_wait(b_, parity, af, st_, tag)) != 0;
       };

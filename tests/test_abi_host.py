@@ -92,6 +92,28 @@ def test_assemble_rejections_match_oracle(kv):
     assert _status(kv.kv_unpack_assemble, cache, short, [2, 3], [5, 6], [0, 1], 64, stream=0) == O.ERR_WIRE_SIZE
 
 
+def test_assemble_random_defects_match_oracle(kv):
+    """600 seeded argument sets (valid states with zero, one or two defects, tests/assemble_cases.py): whenever the
+    oracle's check refuses a set the library refuses it with the same code, before anything is enqueued."""
+    from tests.assemble_cases import random_case
+    s = synth.SHAPES["tiny"]
+    nb = 24
+    cache = _FakeCache(kv, s, nb)
+    page = synth.kv_page_bytes(s)
+    refused = {}
+    for seed in range(600):
+        a = random_case(seed, nb, s.block_size)
+        want = O.check_assemble(nb, s.block_size, a["logical"], a["dst"], a["prefix"], a["n"], a["epoch"], a["expected"])
+        if want == O.OK:
+            continue
+        wire = _FakeBuf(max(len(a["dst"]), 1) * s.n_layers * 2 * page)
+        got = _status(kv.kv_unpack_assemble, cache, wire, a["logical"], a["dst"], a["prefix"], a["n"],
+                      epoch=a["epoch"], expected_epoch=a["expected"], stream=0)
+        assert got == want, (seed, a, got, want)
+        refused[want] = refused.get(want, 0) + 1
+    assert set(refused) == {O.ERR_STALE_EPOCH, O.ERR_BLOCK_RANGE, O.ERR_BLOCK_ALIAS, O.ERR_OVERLAP, O.ERR_GAP}, refused
+
+
 def test_pack_rejections(kv):
     s = synth.SHAPES["tiny"]
     cache = _FakeCache(kv, s, 12)

@@ -62,6 +62,42 @@ def test_pack_unpack_bit_exact_tiny(kv, torch, cache_layout, wire_layout):
     assert np.array_equal(dst.as_logical_numpy(), dst_img)             # pages and canaries, whole cache
 
 
+def test_unpack_assemble_random_cases_against_oracle(kv, torch):
+    """300 seeded migration states (tests/assemble_cases.py: arbitrary arrival order, partly filled last block, empty
+    prefix or empty suffix, and defects of every kind the consistency checks exist for): status, merged table and
+    the whole cache image equal the oracle's, bit for bit; a refused set leaves the cache untouched."""
+    from paper_2608_16477_b200 import KVError
+    from tests.assemble_cases import random_case
+    s = synth.SHAPES["tiny"]
+    nb = 24
+    page = synth.kv_page_bytes(s) // 2
+    rng = np.random.default_rng(77)
+    dst = kv.PagedCache(s, nb, fill=0x5A5A)
+    want_img = np.full((s.n_layers, 2, nb, s.block_size, s.n_kv_heads, s.head_dim), 0x5A5A, dtype=np.uint16)
+    accepted = 0
+    for seed in range(300):
+        a = random_case(seed, nb, s.block_size)
+        n_wire = len(a["dst"])
+        wire_np = rng.integers(0, 65536, (max(n_wire, 1), s.n_layers, 2, page)).astype(np.uint16)
+        wire = _bits_to_torch(torch, wire_np)
+        want_st, want_merged = O.unpack_assemble(want_img, wire_np[:n_wire].reshape(n_wire, s.n_layers, 2, s.block_size,
+                                                                                    s.n_kv_heads, s.head_dim),
+                                                 a["logical"], a["dst"], a["prefix"], a["n"], a["epoch"], a["expected"])
+        try:
+            merged = kv.kv_unpack_assemble(dst, wire, a["logical"], a["dst"], a["prefix"], a["n"], epoch=a["epoch"],
+                                           expected_epoch=a["expected"], wire_bytes=n_wire * s.n_layers * 2 * page * 2)
+            got_st = 0
+        except KVError as e:
+            got_st, merged = e.status, None
+        assert got_st == want_st, (seed, a, got_st, want_st)
+        if want_st == O.OK:
+            accepted += 1
+            assert np.array_equal(merged, want_merged), (seed, a)
+        assert np.array_equal(dst.as_logical_numpy(), want_img), (seed, a)
+    kv.kv_check_copy_status()
+    assert accepted >= 60
+
+
 def test_pack_ragged_and_empty(kv, torch):
     # odd geometry: page of 1 slot x 1 head x 32 dims = 64 bytes; more blocks than one launch carries
     s = synth.ModelShape("odd", n_layers=3, hidden=64, n_q_heads=1, n_kv_heads=1, head_dim=32, ffn=64, vocab=16,
