@@ -454,6 +454,27 @@ def test_scenario_odd_query_group(kv):
         assert error_stats(res["prefill_logits"], lp)["rel_l2"] <= REL_L2
 
 
+@pytest.mark.parametrize("dims", [
+    dict(hidden=264, n_q_heads=6, n_kv_heads=3, head_dim=64, ffn=520, vocab=1001),     # nothing a multiple of a tile
+    dict(hidden=136, n_q_heads=3, n_kv_heads=3, head_dim=128, ffn=200, vocab=333),     # one query head per KV head, d 128
+    dict(hidden=72, n_q_heads=10, n_kv_heads=2, head_dim=64, ffn=40, vocab=50),        # five heads per group, tiny widths
+])
+def test_scenario_awkward_dimensions(kv, dims):
+    """Model dimensions that are multiples of 8 (the interface's only requirement) and of no tile size: every kernel's
+    ragged column and K tails, through the whole path against the oracle (prefix 208 = 13 blocks, resume at 300: above
+    one 128-row tile, a partly filled last block)."""
+    s = synth.ModelShape("awkward", n_layers=2, sharp=True, **dims)
+    ids = synth.token_ids(s, 3, 301)
+    Kref, Vref, logits_ref = oracle_reference(s, 3, ids)
+    res = run_gpu_scenario(kv, s, 3, ids, 208, 300)
+    assert np.array_equal(res["merged"], res["expected_merged"])
+    for name, got, ref in (("K", res["K"], Kref), ("V", res["V"], Vref), ("logits", res["logits"], logits_ref)):
+        st = error_stats(got, ref)
+        assert st["rel_l2"] <= REL_L2 and st["scaled_ok"], (dims, name, st)
+    _, _, lp = oracle_reference(s, 3, ids[:208])
+    assert error_stats(res["prefill_logits"], lp)["rel_l2"] <= REL_L2
+
+
 def test_scenario_tiny_block_major_layer_major_wire(kv):
     s = synth.SHAPES["tiny-sharp"]
     ids = synth.token_ids(s, 0, 161)
