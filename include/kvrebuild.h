@@ -16,7 +16,9 @@
  *     Nothing throws, aborts or prints.
  *   - Pointers named *_dev are DEVICE pointers, *_host are HOST pointers.  All device buffers
  *     (weights, caches, wire buffers, workspaces, logits) are owned by the caller; the library never
- *     allocates or frees device memory.  Host arrays may be reused as soon as a call returns.
+ *     allocates or frees device memory.  Host arrays (pageable or page-locked) may be reused as soon as a
+ *     call returns: the library copies them into page-locked staging slots of its own (host memory, a few
+ *     slots per device that grow to the largest array seen) and transfers from there.
  *   - Work is enqueued on the caller's stream (a cudaStream_t passed as void*); calls do not
  *     synchronise except where stated.  Argument errors are detected on the host before anything is
  *     enqueued, so on a negative status other than KV_ERR_CUDA / KV_ERR_DEVICE no device memory was

@@ -1,7 +1,9 @@
 // C ABI: argument validation on the host, workspace carving and the launch sequences of the four operations.
 #include <algorithm>
 #include <cstdlib>
+#include <atomic>
 #include <cstring>
+#include <mutex>
 #include <string>
 #include <vector>
 
@@ -16,7 +18,7 @@ void set_cuda_error(cudaError_t e, const char *what) {
   (void)cudaGetLastError();
 }
 
-long long g_launches = 0;
+std::atomic<long long> g_launches{0};
 
 int sm_count(int device) {
   static int cached[kMaxDevices] = {};
@@ -27,6 +29,59 @@ int sm_count(int device) {
     cached[device] = n;
   }
   return cached[device];
+}
+
+// ---- page-locked staging of the host arrays of a call (token ids, block tables, per-row metadata) ----
+// A call copies each host array into a page-locked slot owned by the library and enqueues the transfer from there:
+// the caller's array may be reused as soon as the call returns whether it is pageable or page-locked, and the
+// transfer never makes the host wait for earlier work of the stream.  A slot is reused after kStageSlots later
+// uploads on the same device; an event recorded behind its transfer says when that is safe.  Slots grow to the
+// largest array seen and live until the process ends.
+class HostStage {
+ public:
+  int upload(void *dst_dev, const void *src_host, size_t bytes, cudaStream_t st) {
+    if (bytes == 0) return KV_OK;
+    const int device = current_device();
+    if (device < 0) return KV_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu_);
+    Slot &s = slots_[device][next_[device]];
+    next_[device] = (next_[device] + 1) % kStageSlots;
+    if (s.busy) {
+      KV_CUDA(cudaEventSynchronize(s.done));
+      s.busy = false;
+    }
+    if (s.cap < bytes) {
+      if (s.mem != nullptr) KV_CUDA(cudaFreeHost(s.mem));
+      s.mem = nullptr;
+      s.cap = 0;
+      const size_t cap = (bytes + 65535) & ~(size_t)65535;
+      KV_CUDA(cudaHostAlloc(&s.mem, cap, cudaHostAllocPortable));
+      s.cap = cap;
+    }
+    if (s.done == nullptr) KV_CUDA(cudaEventCreateWithFlags(&s.done, cudaEventDisableTiming));
+    memcpy(s.mem, src_host, bytes);
+    KV_CUDA(cudaMemcpyAsync(dst_dev, s.mem, bytes, cudaMemcpyHostToDevice, st));
+    KV_CUDA(cudaEventRecord(s.done, st));
+    s.busy = true;
+    return KV_OK;
+  }
+
+ private:
+  static constexpr int kStageSlots = 16;
+  struct Slot {
+    void *mem = nullptr;
+    size_t cap = 0;
+    cudaEvent_t done = nullptr;
+    bool busy = false;
+  };
+  std::mutex mu_;
+  Slot slots_[kMaxDevices][kStageSlots];
+  int next_[kMaxDevices] = {};
+};
+
+static HostStage &host_stage() {
+  static HostStage *stage = new HostStage();   // never destroyed: page-locked memory must not be freed at exit
+  return *stage;
 }
 
 // ---- optional event profiler: CUDA events around each kernel class, on the caller's stream ----
@@ -476,8 +531,8 @@ int32_t kv_prefill_prefix(kv_model *m, const kv_cache_desc *cache, const int32_t
   // buffers are sized by the context length n_ctx; only the first n_tokens rows are used
   cudaStream_t st = (cudaStream_t)stream;
   KV_CUDA(cudaMemsetAsync(w.status, 0, sizeof(DeviceStatus), st));
-  KV_CUDA(cudaMemcpyAsync(w.ids, token_ids_host, sizeof(int) * n_tokens, cudaMemcpyHostToDevice, st));
-  KV_CUDA(cudaMemcpyAsync(w.table, block_table_host, sizeof(int) * need_blocks, cudaMemcpyHostToDevice, st));
+  KV_TRY(host_stage().upload(w.ids, token_ids_host, sizeof(int) * n_tokens, st));
+  KV_TRY(host_stage().upload(w.table, block_table_host, sizeof(int) * need_blocks, st));
   std::vector<PrefillSegment> segs{{0, n_tokens, logits_out_dev}};
   return prefill_layers(m, make_view(cache), w, n_tokens, pos0, segs, nullptr, nullptr, logits_out_dev != nullptr, st);
 }
@@ -521,8 +576,8 @@ int32_t kv_prefill_prefix_batched(kv_model *m, const kv_cache_desc *cache, int32
   if (workspace_bytes < w.bytes) return KV_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   KV_CUDA(cudaMemsetAsync(w.status, 0, sizeof(DeviceStatus), st));
-  KV_CUDA(cudaMemcpyAsync(w.ids, token_ids_host, sizeof(int) * total, cudaMemcpyHostToDevice, st));
-  KV_CUDA(cudaMemcpyAsync(w.row_meta, row_meta.data(), sizeof(int) * 2 * total, cudaMemcpyHostToDevice, st));
+  KV_TRY(host_stage().upload(w.ids, token_ids_host, sizeof(int) * total, st));
+  KV_TRY(host_stage().upload(w.row_meta, row_meta.data(), sizeof(int) * 2 * total, st));
   return prefill_layers(m, make_view(cache), w, total, 0, segs, w.row_meta, w.row_meta + total, logits_out_dev != nullptr,
                         st);
 }
@@ -550,7 +605,7 @@ int32_t kv_decode_step(kv_model *m, const kv_cache_desc *cache, int32_t token_id
   const int q_dim = d.n_q_heads * d.head_dim;
 
   KV_CUDA(cudaMemsetAsync(w.status, 0, sizeof(DeviceStatus), st));
-  KV_CUDA(cudaMemcpyAsync(w.table, block_table_host, sizeof(int) * need_blocks, cudaMemcpyHostToDevice, st));
+  KV_TRY(host_stage().upload(w.table, block_table_host, sizeof(int) * need_blocks, st));
   {
     ProfScope ps(PROF_DECODE_OTHER, st);
     KV_TRY(rope_table(w.rope, pos, 1, d.head_dim, d.rope_base, st));

@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/kvrebuild.h"
 
 namespace kvr {
@@ -57,8 +59,8 @@ struct DeviceStatus {
 void set_cuda_error(cudaError_t e, const char *what);
 
 // Number of kernels launched by this library so far (host counter, bumped by every launcher).
-extern long long g_launches;
-#define KV_COUNT_LAUNCH() (++::kvr::g_launches)
+extern std::atomic<long long> g_launches;
+#define KV_COUNT_LAUNCH() (::kvr::g_launches.fetch_add(1, std::memory_order_relaxed))
 
 // Kernel classes reported by the optional event profiler (kv_profile_*).
 enum ProfKind {

@@ -153,6 +153,61 @@ def test_chunked_prefill_against_oracle_wide(kv, torch, wide):
     assert st["rel_l2"] <= exact_bound(s.n_layers), st
 
 
+# ------------------------------------------------------------------ host arrays belong to the caller again on return
+def test_host_arrays_may_be_overwritten_as_soon_as_a_call_returns(kv, torch):
+    """Token ids and block tables handed over in page-locked memory, with the stream still busy when the call returns,
+    are overwritten at once with other (valid) values: prefill, batched prefill and decode step must have taken their
+    own copy.  The reference results come from the same calls with untouched arrays."""
+    s, head, lw, model = _tiny_model(kv, "tiny", 11)
+    n = 96
+    ids = synth.token_ids(s, 11, n + 1)
+    table = synth.block_permutation(12, 64)[: n // 16 + 1]
+    other_ids = synth.token_ids(s, 13, n + 1)
+    other_table = synth.block_permutation(14, 64)[: n // 16 + 1]
+    busy = torch.empty(1 << 30, dtype=torch.uint8, device="cuda")
+
+    def pinned(a):
+        t = torch.from_numpy(np.asarray(a, dtype=np.int32).copy()).pin_memory()
+        return t, t.numpy()
+
+    def run(overwrite):
+        cache = kv.PagedCache(s, 64, fill=0)
+        lg = torch.zeros(3, s.vocab, dtype=torch.float32, device="cuda")
+        keep = []
+        def hand_over(a, b):
+            t, view = pinned(a)
+            keep.append(t)
+            return view, np.asarray(b, dtype=np.int32)
+        def clobber(*pairs):
+            if overwrite:
+                for view, repl in pairs:
+                    view[:] = repl
+        def delay():                                   # a few milliseconds of work ahead of the call in the stream
+            for _ in range(12):
+                kv.kv_fill_pattern(busy, busy.numel(), seed=1)
+        i1, t1 = hand_over(ids[:n], other_ids[:n]), hand_over(table[: n // 16], other_table[: n // 16])
+        delay()
+        kv.kv_prefill_prefix(model, cache, i1[0], t1[0], logits_out=lg[0])
+        clobber(i1, t1)
+        t2 = hand_over(table, other_table)
+        delay()
+        kv.kv_decode_step(model, cache, int(ids[n]), n, t2[0], lg[1])
+        clobber(t2)
+        # the batched form into other pages of the same cache
+        free = np.setdiff1d(np.arange(64), table)[: n // 16]
+        i3, t3 = hand_over(ids[:n], other_ids[:n]), hand_over(free, free[::-1].copy())
+        delay()
+        kv.kv_prefill_prefix_batched(model, cache, [i3[0]], [t3[0]], logits_out=lg[2:3])
+        clobber(i3, t3)
+        torch.cuda.synchronize()
+        return cache.data.clone(), lg.clone()
+
+    ref_cache, ref_lg = run(False)
+    got_cache, got_lg = run(True)
+    assert bool(ref_cache.any()) and torch.equal(got_cache, ref_cache)
+    assert torch.equal(got_lg, ref_lg)
+
+
 # ------------------------------------------------------------------ "without suffix migration"
 @pytest.mark.parametrize("name", ["tiny", "tiny-sharp"])
 def test_suffix_recomputed_at_target_tiny(kv, torch, name):
