@@ -275,7 +275,7 @@ int32_t kv_op_paged_attention(const float *q_dev, int32_t n_q_heads, const kv_ca
  *    KV_NOALLOC_SCRATCH_BYTES, otherwise KV_ERR_WORKSPACE is returned and nothing is launched
  *    (64 query heads of dimension 128 fit up to 16,128 context tokens).
  *  - The call never allocates or frees memory.  Its first call on a device looks up the array's device
- *    address (once per device); make that first call before starting any stream capture.
+ *    address (once per device).
  *  - All calls on a device share the one array and it keeps whatever the last call left there.  A call
  *    writes every partial it later reads, so stale contents are harmless, but two calls whose kernels can
  *    overlap on the GPU (different streams) race on it: serialise them. */
