@@ -243,7 +243,8 @@ int32_t kv_op_gemv(const void *w_dev, const float *x_dev, int32_t n, int32_t k, 
 int32_t kv_gemm_plan(int32_t m, int32_t n, int32_t mode, int32_t head_dim, int32_t *cta_pair_out,
                      int32_t *tile_width_out);
 
-/* RMSNorm of fp32 rows x [rows, dim] with bf16 gain -> bf16 out [rows, dim]. */
+/* RMSNorm of fp32 rows x [rows, dim] with bf16 gain -> bf16 out [rows, dim].  dim a multiple of 4; x_dev 16-byte,
+ * gain_dev and out_dev 8-byte aligned. */
 int32_t kv_op_rmsnorm(const float *x_dev, const void *gain_dev, int32_t rows, int32_t dim, float eps,
                       void *out_dev, void *stream);
 

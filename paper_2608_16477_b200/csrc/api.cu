@@ -337,6 +337,8 @@ int32_t kv_model_create(const kv_model_desc *desc, const kv_weights *w, kv_model
   if (!w->embed_dev || !w->lm_head_dev || !w->final_norm_dev || !w->attn_norm_dev || !w->w_qkv_dev || !w->w_o_dev ||
       !w->ffn_norm_dev || !w->w_gate_up_dev || !w->w_down_dev)
     return KV_ERR_ARG;
+  if (((uintptr_t)w->embed_dev & 15) || ((uintptr_t)w->lm_head_dev & 15) || ((uintptr_t)w->final_norm_dev & 15))
+    return KV_ERR_ARG;
   kv_model *m = new kv_model();
   m->d = d;
   m->embed = (const bf16 *)w->embed_dev;
@@ -756,6 +758,8 @@ int32_t kv_op_rmsnorm(const float *x_dev, const void *gain_dev, int32_t rows, in
                       void *stream) {
   if (x_dev == nullptr || gain_dev == nullptr || out_dev == nullptr || rows < 0 || dim <= 0 || dim % 4 != 0)
     return KV_ERR_ARG;
+  // the kernel reads x as float4 and gain as 4 x bf16, and writes 4 x bf16 at a time
+  if (((uintptr_t)x_dev & 15) || ((uintptr_t)gain_dev & 7) || ((uintptr_t)out_dev & 7)) return KV_ERR_ARG;
   return rmsnorm_rows(x_dev, (const bf16 *)gain_dev, rows, dim, eps, (bf16 *)out_dev, (cudaStream_t)stream);
 }
 

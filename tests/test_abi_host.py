@@ -140,6 +140,15 @@ def test_prefill_and_decode_rejections(kv):
     bad = ModelDesc(s.n_layers, s.hidden, 3, 2, s.head_dim, s.ffn, s.vocab, 1e6, 1e-6)
     h2 = C.c_void_p()
     assert lib.kv_model_create(C.byref(bad), C.byref(w), C.byref(h2)) == O.ERR_SHAPE
+    # weight pointers are read as 16-byte vectors: a misaligned one is refused when the handle is created
+    odd = (C.c_void_p * s.n_layers)(*[fake + 8] * s.n_layers)
+    podd = C.cast(odd, C.POINTER(C.c_void_p))
+    for wbad in (Weights(fake + 8, fake, fake, parr, parr, parr, parr, parr, parr),
+                 Weights(fake, fake + 2, fake, parr, parr, parr, parr, parr, parr),
+                 Weights(fake, fake, fake + 4, parr, parr, parr, parr, parr, parr),
+                 Weights(fake, fake, fake, parr, podd, parr, parr, parr, parr),
+                 Weights(fake, fake, fake, parr, parr, parr, parr, parr, podd)):
+        assert lib.kv_model_create(C.byref(d), C.byref(wbad), C.byref(h2)) == O.ERR_ARG
 
     class M:
         handle = h
@@ -220,6 +229,16 @@ def test_single_kernel_entry_points_reject_misaligned_arguments(kv):
     assert lib.kv_op_attention_prefill(a + 8, 10, 0, 8, 2, 128, None, 0, None, o, None, 0) == O.ERR_ARG
     assert lib.kv_op_attention_prefill(a, 10, 8, 8, 2, 128, C.byref(good.desc), 0, table, o, None, 0) == O.ERR_SPLIT_UNALIGNED
     assert lib.kv_op_attention_prefill(a, 10, 16, 8, 2, 128, None, 0, table, o, None, 0) == O.ERR_ARG
+    # RMSNorm reads float4 and writes four bf16 at a time; the matrix-vector product reads 16-byte vectors
+    fp = lambda v: C.cast(v, C.POINTER(C.c_float))
+    eps = C.c_float(1e-6)
+    assert lib.kv_op_rmsnorm(fp(a + 8), w, 4, 64, eps, o, 0) == O.ERR_ARG
+    assert lib.kv_op_rmsnorm(fp(a), w + 4, 4, 64, eps, o, 0) == O.ERR_ARG
+    assert lib.kv_op_rmsnorm(fp(a), w, 4, 64, eps, o + 4, 0) == O.ERR_ARG
+    assert lib.kv_op_rmsnorm(fp(a), w, 4, 66, eps, o, 0) == O.ERR_ARG
+    assert lib.kv_op_gemv(w + 8, fp(a), 16, 64, 0, None, eps, fp(r), 0) == O.ERR_ARG
+    assert lib.kv_op_gemv(w, fp(a + 4), 16, 64, 0, None, eps, fp(r), 0) == O.ERR_ARG
+    assert lib.kv_op_gemv(w, fp(a), 16, 60, 0, None, eps, fp(r), 0) == O.ERR_SHAPE
 
 
 def test_gemm_plan_query(kv):
