@@ -26,8 +26,10 @@ RMSNorm/SwiGLU closed forms, RoPE invariants, brute-force loop attention on tiny
 torch SDPA as a black-box library cross-check, causality between the full-sequence, the
 chunk-by-chunk (cached-prefix) and the incremental code paths, the fp32 library matmul against
 the fp64 one and against an error bound, the bf16 storage points against the library cast at
-each of them, pack/unpack by a five-deep byte loop.
-Parity unpinned: fidelity to real Qwen3/Llama checkpoints (no weights are available).
+each of them, pack/unpack by a five-deep byte loop,
+the whole forward (K, V and all logits) against the library's Llama decoder loaded with the same weights.
+Every function of this module has a pin.  Outside what a pin can reach: agreement with the published
+Qwen3/Llama checkpoints (no weights are available; the architecture is pinned, trained values are not involved).
 """
 from __future__ import annotations
 
