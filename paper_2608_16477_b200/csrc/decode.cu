@@ -290,27 +290,34 @@ __global__ void __launch_bounds__(kPaSplitKeys, 2) paged_attention_split_kernel(
   const int j0 = split * kPaSplitKeys;
   const int n_keys = min(n_ctx - j0, kPaSplitKeys);
 
-  // this thread's key (rows past the end repeat the last key: finite data, masked below)
+  // K and V rows of the split into shared memory.  A warp copies its 32 rows (keys 32w..32w+31, the ones its MMAs
+  // read) 32 / CH rows at a time: CH consecutive lanes cover one row's CH 16-byte chunks, so every instruction
+  // moves whole rows (contiguous 2 D bytes each) instead of one chunk of 32 different rows.  Rows past the end
+  // repeat the last key (finite data, masked below).
   {
-    const int jk = j0 + min(tid, n_keys - 1);
-    const long long row_off = ((long long)(jk % cache.block_size) * cache.n_kv_heads + g) * D;
-    const int blk = block_table[jk / cache.block_size];
-    const bf16 *kp = reinterpret_cast<const bf16 *>(cache.page(layer, 0, blk)) + row_off;
-    const bf16 *vp = reinterpret_cast<const bf16 *>(cache.page(layer, 1, blk)) + row_off;
-    const uint32_t kd = (uint32_t)__cvta_generic_to_shared(k_tile + tid * RB);
-    const uint32_t vd = (uint32_t)__cvta_generic_to_shared(v_tile + tid * RB);
+    constexpr int RPI = 32 / CH;              // rows per instruction
+    const int sub = lane / CH, c = lane % CH;
+    const int bsz = cache.block_size;
+    // lane l looks up the page and the slot of the warp's row l once; the copy loop fetches them by shuffle
+    const int jk = min(j0 + warp * 32 + lane, j0 + n_keys - 1);
+    const int my_blk = block_table[jk / bsz];
+    const int my_slot = jk % bsz;
 #pragma unroll
-    for (int c = 0; c < CH; ++c) {
-      const uint32_t pc = (uint32_t)((c & ~7) | ((c ^ tid) & 7)) * 16;
-      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(kd + pc), "l"(kp + c * 8) : "memory");
-    }
-    asm volatile("cp.async.commit_group;" ::: "memory");
+    for (int kv = 0; kv < 2; ++kv) {
+      const uint32_t tile = (uint32_t)__cvta_generic_to_shared(kv == 0 ? k_tile : v_tile);
 #pragma unroll
-    for (int c = 0; c < CH; ++c) {
-      const uint32_t pc = (uint32_t)((c & ~7) | ((c ^ tid) & 7)) * 16;
-      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(vd + pc), "l"(vp + c * 8) : "memory");
+      for (int i = 0; i < CH; ++i) {
+        const int rw = i * RPI + sub;                        // row inside the warp's 32
+        const int r = warp * 32 + rw;                        // row of the tile
+        const int blk = __shfl_sync(0xffffffffu, my_blk, rw);
+        const int slot = __shfl_sync(0xffffffffu, my_slot, rw);
+        const bf16 *src = reinterpret_cast<const bf16 *>(cache.page(layer, kv, blk)) +
+                          ((long long)slot * cache.n_kv_heads + g) * D + c * 8;
+        const uint32_t pc = (uint32_t)((c & ~7) | ((c ^ r) & 7)) * 16;
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(tile + r * RB + pc), "l"(src) : "memory");
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
     }
-    asm volatile("cp.async.commit_group;" ::: "memory");
   }
   const uint32_t k_s = (uint32_t)__cvta_generic_to_shared(k_tile);
   const uint32_t v_s = (uint32_t)__cvta_generic_to_shared(v_tile);
