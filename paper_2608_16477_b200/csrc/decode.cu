@@ -221,9 +221,9 @@ int gemv_qkv_rope(const bf16 *w_qkv, const float *x, const bf16 *gain, float eps
 // ---- paged decode attention ---------------------------------------------------------------
 // Partial record per (q head, split): m, l, acc[d].
 // One CTA of 128 threads per (KV head, 128-key split), serving every query head of the group so each K/V
-// row is read from HBM once.  Thread t copies the K row and the V row of key t into shared memory with
-// 16-byte cp.async (everything in flight at once; 16-byte chunks XOR-swizzled by the row so that ldmatrix is
-// conflict-free).  The contractions run on mma.sync m16n8k16 (a 16-row tile is the natural size for the 8 to
+// row is read from HBM once.  The K and V rows of the split go to shared memory with 16-byte cp.async, d/8
+// consecutive lanes per row (everything in flight at once; 16-byte chunks XOR-swizzled by the row so that ldmatrix
+// is conflict-free).  The contractions run on mma.sync m16n8k16 (a 16-row tile is the natural size for the 8 to
 // 16 query heads of a group; the 128-row tcgen05 tile would be nine tenths padding):
 //   S = Q K^T   warp w owns keys 32w..32w+31; Q (fp32) is split into a bf16 high and low part, so the scores
 //               keep fp32-level accuracy at the cost of a second MMA;
