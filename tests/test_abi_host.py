@@ -254,3 +254,20 @@ def test_gemm_plan_query(kv):
         kv.kv_gemm_plan(4096, 10240, 3, head_dim=96)
     with pytest.raises(KVError):
         kv.kv_gemm_plan(0, 10240, 1)
+
+
+def test_header_is_plain_c_and_a_c_program_links(kv, tmp_path):
+    """The header compiles as strict C99 (no C++, no torch types) and a C program linked against the library runs the
+    host-only entry points."""
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    assert gcc, "gcc is part of the build environment"
+    libdir = os.path.dirname(kv.lib_path())
+    exe = str(tmp_path / "abi_c_consumer")
+    subprocess.run([gcc, "-std=c99", "-pedantic", "-Wall", "-Wextra", "-Werror", "-I" + os.path.join(ROOT, "include"),
+                    os.path.join(ROOT, "tests", "abi_c_consumer.c"), "-o", exe, "-L" + libdir, "-lkvrebuild",
+                    "-Wl,-rpath," + libdir], check=True, capture_output=True, text=True)
+    run = subprocess.run([exe], capture_output=True, text=True)
+    assert run.returncode == 0, (run.returncode, run.stdout, run.stderr)
+    assert run.stdout.startswith("t_w=")
