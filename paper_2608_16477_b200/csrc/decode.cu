@@ -282,24 +282,29 @@ __global__ void __launch_bounds__(kPaSplitKeys, 2) paged_attention_split_kernel(
   uint8_t *k_tile = pa_smem;                                  // [keys][D] bf16, swizzled
   uint8_t *v_tile = pa_smem + kPaSplitKeys * RB;
   float *o_red = reinterpret_cast<float *>(pa_smem + 2 * kPaSplitKeys * RB);   // [NW][kPaRows][D] partial O
-  __shared__ float wmax_s[NW][kPaRows], wsum_s[NW][kPaRows];
-  const int g = blockIdx.x, split = blockIdx.y, n_splits = gridDim.y;
+  __shared__ float wmax_s[NW][kPaRows], wsum_s[NW][kPaRows], run_max_s[kPaRows];
+  // CTA (g, part) walks the 128-key tiles [t_begin, t_end) of KV head g: one tile when the context has no more tiles
+  // than the grid has parts (the launcher asks for two CTAs per SM), several consecutive ones for longer contexts,
+  // carried by a running maximum, running sums and one output accumulator (one partial record per part either way).
+  const int g = blockIdx.x, part = blockIdx.y, n_parts = gridDim.y;
+  const int n_tiles = (n_ctx + kPaSplitKeys - 1) / kPaSplitKeys;
+  const int t_begin = (int)((long long)part * n_tiles / n_parts);
+  const int t_end = (int)((long long)(part + 1) * n_tiles / n_parts);
+  const bool one_tile = t_end - t_begin == 1;
   const int group = n_q_heads / cache.n_kv_heads;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float scale = rsqrtf((float)D);
-  const int j0 = split * kPaSplitKeys;
-  const int n_keys = min(n_ctx - j0, kPaSplitKeys);
 
-  // K and V rows of the split into shared memory.  A warp copies its 32 rows (keys 32w..32w+31, the ones its MMAs
+  // K and V rows of a tile into shared memory.  A warp copies its 32 rows (keys 32w..32w+31, the ones its MMAs
   // read) 32 / CH rows at a time: CH consecutive lanes cover one row's CH 16-byte chunks, so every instruction
   // moves whole rows (contiguous 2 D bytes each) instead of one chunk of 32 different rows.  Rows past the end
-  // repeat the last key (finite data, masked below).
-  {
+  // repeat the last key (finite data, masked below).  Two commit groups: K first, then V.
+  auto load_tile = [&](int t) {
     constexpr int RPI = 32 / CH;              // rows per instruction
     const int sub = lane / CH, c = lane % CH;
     const int bsz = cache.block_size;
     // lane l looks up the page and the slot of the warp's row l once; the copy loop fetches them by shuffle
-    const int jk = min(j0 + warp * 32 + lane, j0 + n_keys - 1);
+    const int jk = min(t * kPaSplitKeys + warp * 32 + lane, n_ctx - 1);
     const int my_blk = block_table[jk / bsz];
     const int my_slot = jk % bsz;
 #pragma unroll
@@ -318,11 +323,12 @@ __global__ void __launch_bounds__(kPaSplitKeys, 2) paged_attention_split_kernel(
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
     }
-  }
+  };
+  load_tile(t_begin);
   const uint32_t k_s = (uint32_t)__cvta_generic_to_shared(k_tile);
   const uint32_t v_s = (uint32_t)__cvta_generic_to_shared(v_tile);
   const int r0 = lane >> 2, cq = (lane & 3) * 2;       // fragment row (and row + 8), first of two columns
-  const int wk0 = warp * 32;                           // this warp's keys inside the split
+  const int wk0 = warp * 32;                           // this warp's keys inside a tile
 
   for (int h0 = 0; h0 < group; h0 += kPaRows) {
     const int nh = min(kPaRows, group - h0);
@@ -344,84 +350,112 @@ __global__ void __launch_bounds__(kPaSplitKeys, 2) paged_attention_split_kernel(
         split_pair(b2.x * sb, b2.y * sb, qh[ks][3], ql[ks][3]);
       }
     }
-    if (h0 == 0) asm volatile("cp.async.wait_group 1;" ::: "memory");      // K rows have landed
-    __syncthreads();      // (also: the previous pass no longer reads o_red and the row statistics)
-    // ---- S = Q K^T for this warp's 32 keys: 4 n-tiles of 8 keys
-    float sc[4][4];
-#pragma unroll
-    for (int nt = 0; nt < 4; ++nt) {
-#pragma unroll
-      for (int i = 0; i < 4; ++i) sc[nt][i] = 0.f;
-      const int krow = wk0 + nt * 8 + (lane & 7);
-#pragma unroll
-      for (int ks = 0; ks < KS; ks += 2) {
-        const int chunk = ks * 2 + (lane >> 3);
-        uint32_t bfr[4];
-        ldmatrix_x4(k_s + krow * RB + (uint32_t)((chunk & ~7) | ((chunk ^ krow) & 7)) * 16, bfr);
-        mma_bf16_16816(sc[nt], qh[ks], bfr[0], bfr[1]);
-        mma_bf16_16816(sc[nt], ql[ks], bfr[0], bfr[1]);
-        mma_bf16_16816(sc[nt], qh[ks + 1], bfr[2], bfr[3]);
-        mma_bf16_16816(sc[nt], ql[ks + 1], bfr[2], bfr[3]);
-      }
-    }
-    // mask keys past the end, row maxima over this warp's keys
-    float mx0 = -FLT_MAX, mx1 = -FLT_MAX;
-#pragma unroll
-    for (int nt = 0; nt < 4; ++nt) {
-      const int key = wk0 + nt * 8 + cq;
-      if (key >= n_keys) sc[nt][0] = sc[nt][2] = -FLT_MAX;
-      if (key + 1 >= n_keys) sc[nt][1] = sc[nt][3] = -FLT_MAX;
-      mx0 = fmaxf(mx0, fmaxf(sc[nt][0], sc[nt][1]));
-      mx1 = fmaxf(mx1, fmaxf(sc[nt][2], sc[nt][3]));
-    }
-    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-    if ((lane & 3) == 0) {
-      wmax_s[warp][r0] = mx0;
-      wmax_s[warp][r0 + 8] = mx1;
-    }
-    if (h0 == 0) asm volatile("cp.async.wait_group 0;" ::: "memory");      // V rows have landed
-    __syncthreads();
-    mx0 = wmax_s[0][r0];
-    mx1 = wmax_s[0][r0 + 8];
-#pragma unroll
-    for (int w = 1; w < NW; ++w) {
-      mx0 = fmaxf(mx0, wmax_s[w][r0]);
-      mx1 = fmaxf(mx1, wmax_s[w][r0 + 8]);
-    }
-    // ---- probabilities (A fragments, high + low) and O = P V over this warp's two 16-key steps
-    float sum0 = 0.f, sum1 = 0.f;
-    uint32_t ph[2][4], pl[2][4];
-#pragma unroll
-    for (int nt = 0; nt < 4; ++nt) {
-      const float p0 = __expf(sc[nt][0] - mx0), p1 = __expf(sc[nt][1] - mx0);     // masked scores give 0
-      const float p2 = __expf(sc[nt][2] - mx1), p3 = __expf(sc[nt][3] - mx1);
-      sum0 += p0 + p1;
-      sum1 += p2 + p3;
-      split_pair(p0, p1, ph[nt >> 1][(nt & 1) * 2], pl[nt >> 1][(nt & 1) * 2]);
-      split_pair(p2, p3, ph[nt >> 1][(nt & 1) * 2 + 1], pl[nt >> 1][(nt & 1) * 2 + 1]);
-    }
+    // running state of rows r0 and r0 + 8: the maximum (the same in every warp), this lane's share of the row sums
+    // and the warp's output accumulator over its own keys of every tile
+    float run0 = -FLT_MAX, run1 = -FLT_MAX, sum0 = 0.f, sum1 = 0.f;
     float oc[NT][4];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
       for (int i = 0; i < 4; ++i) oc[nt][i] = 0.f;
+
+    for (int t = t_begin; t < t_end; ++t) {
+      const int n_keys = min(n_ctx - t * kPaSplitKeys, kPaSplitKeys);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");      // K rows have landed
+      __syncthreads();      // (also: the previous tile or pass no longer reads the row statistics and o_red)
+      // ---- S = Q K^T for this warp's 32 keys: 4 n-tiles of 8 keys
+      float sc[4][4];
 #pragma unroll
-    for (int kk = 0; kk < 2; ++kk) {
-      const int vrow = wk0 + kk * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
+      for (int nt = 0; nt < 4; ++nt) {
 #pragma unroll
-      for (int nt = 0; nt < NT; nt += 2) {
-        const int chunk = nt + (lane >> 4);
-        uint32_t bfr[4];
-        ldmatrix_x4_trans(v_s + vrow * RB + (uint32_t)((chunk & ~7) | ((chunk ^ vrow) & 7)) * 16, bfr);
-        mma_bf16_16816(oc[nt], ph[kk], bfr[0], bfr[1]);
-        mma_bf16_16816(oc[nt], pl[kk], bfr[0], bfr[1]);
-        mma_bf16_16816(oc[nt + 1], ph[kk], bfr[2], bfr[3]);
-        mma_bf16_16816(oc[nt + 1], pl[kk], bfr[2], bfr[3]);
+        for (int i = 0; i < 4; ++i) sc[nt][i] = 0.f;
+        const int krow = wk0 + nt * 8 + (lane & 7);
+#pragma unroll
+        for (int ks = 0; ks < KS; ks += 2) {
+          const int chunk = ks * 2 + (lane >> 3);
+          uint32_t bfr[4];
+          ldmatrix_x4(k_s + krow * RB + (uint32_t)((chunk & ~7) | ((chunk ^ krow) & 7)) * 16, bfr);
+          mma_bf16_16816(sc[nt], qh[ks], bfr[0], bfr[1]);
+          mma_bf16_16816(sc[nt], ql[ks], bfr[0], bfr[1]);
+          mma_bf16_16816(sc[nt], qh[ks + 1], bfr[2], bfr[3]);
+          mma_bf16_16816(sc[nt], ql[ks + 1], bfr[2], bfr[3]);
+        }
+      }
+      // mask keys past the end, row maxima over this warp's keys
+      float mx0 = -FLT_MAX, mx1 = -FLT_MAX;
+#pragma unroll
+      for (int nt = 0; nt < 4; ++nt) {
+        const int key = wk0 + nt * 8 + cq;
+        if (key >= n_keys) sc[nt][0] = sc[nt][2] = -FLT_MAX;
+        if (key + 1 >= n_keys) sc[nt][1] = sc[nt][3] = -FLT_MAX;
+        mx0 = fmaxf(mx0, fmaxf(sc[nt][0], sc[nt][1]));
+        mx1 = fmaxf(mx1, fmaxf(sc[nt][2], sc[nt][3]));
+      }
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+      if ((lane & 3) == 0) {
+        wmax_s[warp][r0] = mx0;
+        wmax_s[warp][r0 + 8] = mx1;
+      }
+      asm volatile("cp.async.wait_group 0;" ::: "memory");      // V rows have landed
+      __syncthreads();
+      mx0 = run0;
+      mx1 = run1;
+#pragma unroll
+      for (int w = 0; w < NW; ++w) {
+        mx0 = fmaxf(mx0, wmax_s[w][r0]);
+        mx1 = fmaxf(mx1, wmax_s[w][r0 + 8]);
+      }
+      // what the earlier tiles of this part left is brought to the new maximum (nothing to do for the first tile:
+      // sums and accumulator are zero)
+      if (t > t_begin) {
+        const float f0 = __expf(run0 - mx0), f1 = __expf(run1 - mx1);
+        sum0 *= f0;
+        sum1 *= f1;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          oc[nt][0] *= f0;
+          oc[nt][1] *= f0;
+          oc[nt][2] *= f1;
+          oc[nt][3] *= f1;
+        }
+      }
+      run0 = mx0;
+      run1 = mx1;
+      // ---- probabilities (A fragments, high + low) and O += P V over this warp's two 16-key steps
+      uint32_t ph[2][4], pl[2][4];
+#pragma unroll
+      for (int nt = 0; nt < 4; ++nt) {
+        const float p0 = __expf(sc[nt][0] - mx0), p1 = __expf(sc[nt][1] - mx0);     // masked scores give 0
+        const float p2 = __expf(sc[nt][2] - mx1), p3 = __expf(sc[nt][3] - mx1);
+        sum0 += p0 + p1;
+        sum1 += p2 + p3;
+        split_pair(p0, p1, ph[nt >> 1][(nt & 1) * 2], pl[nt >> 1][(nt & 1) * 2]);
+        split_pair(p2, p3, ph[nt >> 1][(nt & 1) * 2 + 1], pl[nt >> 1][(nt & 1) * 2 + 1]);
+      }
+#pragma unroll
+      for (int kk = 0; kk < 2; ++kk) {
+        const int vrow = wk0 + kk * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
+#pragma unroll
+        for (int nt = 0; nt < NT; nt += 2) {
+          const int chunk = nt + (lane >> 4);
+          uint32_t bfr[4];
+          ldmatrix_x4_trans(v_s + vrow * RB + (uint32_t)((chunk & ~7) | ((chunk ^ vrow) & 7)) * 16, bfr);
+          mma_bf16_16816(oc[nt], ph[kk], bfr[0], bfr[1]);
+          mma_bf16_16816(oc[nt], pl[kk], bfr[0], bfr[1]);
+          mma_bf16_16816(oc[nt + 1], ph[kk], bfr[2], bfr[3]);
+          mma_bf16_16816(oc[nt + 1], pl[kk], bfr[2], bfr[3]);
+        }
+      }
+      // the next tile of this pass, or the first tile again for the next pass of heads (a single tile stays where it is)
+      if (!one_tile && (t + 1 < t_end || h0 + kPaRows < group)) {
+        __syncthreads();      // every warp is done with this tile's K and V
+        load_tile(t + 1 < t_end ? t + 1 : t_begin);
       }
     }
+    // ---- the four warps' shares of O and of the row sums meet in shared memory
     sum0 += __shfl_xor_sync(0xffffffffu, sum0, 1);
     sum0 += __shfl_xor_sync(0xffffffffu, sum0, 2);
     sum1 += __shfl_xor_sync(0xffffffffu, sum1, 1);
@@ -429,6 +463,10 @@ __global__ void __launch_bounds__(kPaSplitKeys, 2) paged_attention_split_kernel(
     if ((lane & 3) == 0) {
       wsum_s[warp][r0] = sum0;
       wsum_s[warp][r0 + 8] = sum1;
+      if (warp == 0) {
+        run_max_s[r0] = run0;
+        run_max_s[r0 + 8] = run1;
+      }
     }
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
@@ -443,16 +481,13 @@ __global__ void __launch_bounds__(kPaSplitKeys, 2) paged_attention_split_kernel(
       float a = 0.f;
 #pragma unroll
       for (int w = 0; w < NW; ++w) a += o_red[(long long)(w * kPaRows + h) * D + c];
-      float *rec = partial + ((long long)(g * group + h0 + h) * n_splits + split) * (D + 2);
+      float *rec = partial + ((long long)(g * group + h0 + h) * n_parts + part) * (D + 2);
       rec[2 + c] = a;
       if (c == 0) {
-        float l = 0.f, m = wmax_s[0][h];
+        float l = 0.f;
 #pragma unroll
-        for (int w = 0; w < NW; ++w) {
-          l += wsum_s[w][h];
-          m = fmaxf(m, wmax_s[w][h]);
-        }
-        rec[0] = m;
+        for (int w = 0; w < NW; ++w) l += wsum_s[w][h];
+        rec[0] = run_max_s[h];
         rec[1] = l;
       }
     }
@@ -496,13 +531,16 @@ __global__ void __launch_bounds__(128) paged_attention_merge_kernel(const float 
 
 int paged_attention(const float *q, int n_q_heads, CacheView cache, int layer, const int *block_table_dev,
                     int n_ctx, void *scratch, float *out, cudaStream_t st) {
-  const int splits = pa_splits(n_ctx);
-  if (splits > kPaMergeMaxSplits) return KV_ERR_SHAPE;   // 262,144 context tokens
-  const dim3 grid(cache.n_kv_heads, splits);
-  float *partial = (float *)scratch;
-  static bool attr_set[kMaxDevices] = {};
   const int device = current_device();
   if (device < 0) return KV_ERR_CUDA;
+  // one part per 128-key tile up to two CTAs per SM; longer contexts give a part several consecutive tiles
+  const int tiles = pa_splits(n_ctx);
+  int parts = 2 * sm_count(device) / cache.n_kv_heads;
+  parts = parts < 1 ? 1 : (parts > kPaMergeMaxSplits ? kPaMergeMaxSplits : parts);
+  if (parts > tiles) parts = tiles;
+  const dim3 grid(cache.n_kv_heads, parts);
+  float *partial = (float *)scratch;
+  static bool attr_set[kMaxDevices] = {};
   if (!attr_set[device]) {
     KV_CUDA(cudaFuncSetAttribute(paged_attention_split_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  pa_smem_bytes(64)));
@@ -520,7 +558,7 @@ int paged_attention(const float *q, int n_q_heads, CacheView cache, int layer, c
     return KV_ERR_SHAPE;
   KV_COUNT_LAUNCH();
   KV_CUDA(cudaGetLastError());
-  paged_attention_merge_kernel<<<n_q_heads, 128, 0, st>>>(partial, splits, cache.head_dim, out);
+  paged_attention_merge_kernel<<<n_q_heads, 128, 0, st>>>(partial, parts, cache.head_dim, out);
   KV_COUNT_LAUNCH();
   KV_CUDA(cudaGetLastError());
   return KV_OK;

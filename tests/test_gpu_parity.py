@@ -378,15 +378,24 @@ def test_attention_prefill_long_context_sampled_rows(kv, torch):
         assert st["max_abs"] <= MAX_ABS and st["rel_l2"] <= REL_L2, (r0, st)
 
 
-@pytest.mark.parametrize("n_ctx,hq,hkv,d", [(777, 8, 2, 128), (1, 4, 2, 64), (128, 16, 1, 128), (129, 8, 1, 64),
-                                            (300, 40, 1, 128), (4609, 64, 8, 128), (20011, 8, 1, 128)])
-def test_paged_decode_attention(kv, torch, n_ctx, hq, hkv, d):
+@pytest.mark.parametrize("n_ctx,hq,hkv,d,ramp", [
+    (777, 8, 2, 128, 0), (1, 4, 2, 64, 0), (128, 16, 1, 128, 0), (129, 8, 1, 64, 0), (300, 40, 1, 128, 0),
+    (4609, 64, 8, 128, 0), (20011, 8, 1, 128, 0),
+    # more 128-key tiles than the grid has parts (two CTAs per SM over the KV heads): a CTA walks several tiles with a
+    # running maximum; `ramp` makes the scores grow (+) or shrink (-) along the context so that maximum keeps moving
+    (4737, 16, 8, 128, 0), (9000, 16, 8, 128, 3), (20011, 32, 8, 64, -3), (7000, 160, 8, 64, 2), (33000, 8, 4, 128, 1)])
+def test_paged_decode_attention(kv, torch, n_ctx, hq, hkv, d, ramp):
     """One query position against a paged context: a single key, exactly one 128-key split, one key past it, many
-    splits; groups of 2 to 40 query heads per KV head (more than the 16 rows one pass of the kernel serves)."""
+    splits, several tiles per CTA; groups of 2 to 40 query heads per KV head (more than the 16 rows one pass of the
+    kernel serves)."""
     s = synth.ModelShape("pa", n_layers=2, hidden=64, n_q_heads=hq, n_kv_heads=hkv, head_dim=d, ffn=64, vocab=16)
     nb = -(-n_ctx // 16) + 7
     rng = np.random.default_rng(8 + n_ctx)
-    K = synth.bf16_round_f32(rng.standard_normal((2, n_ctx, hkv, d), dtype=np.float32))
+    K = rng.standard_normal((2, n_ctx, hkv, d), dtype=np.float32)
+    if ramp:
+        pos = np.arange(n_ctx, dtype=np.float32) / n_ctx
+        K *= (1.0 + abs(ramp) * (pos if ramp > 0 else 1.0 - pos))[None, :, None, None]
+    K = synth.bf16_round_f32(K)
     V = synth.bf16_round_f32(rng.standard_normal((2, n_ctx, hkv, d), dtype=np.float32))
     img = O.new_cache(2, nb, 16, hkv, d)
     table = synth.block_permutation(9, nb)[: -(-n_ctx // 16)]
