@@ -472,7 +472,8 @@ def run_ours(args):
     legs = np.array([[ev[0].elapsed_time(ev[1]), ev[4].elapsed_time(ev[5]), ev[1].elapsed_time(ev[2]),
                       ev[2].elapsed_time(ev[3])] for ev in e2e_marks]).mean(axis=0)
 
-    # prefix-length sweep of the same shape (K/V-only prefill, 3 timed calls each after one warm-up call)
+    # prefix-length sweep of the same shape (K/V-only prefill, 3 timed calls each after one warm-up call; then the
+    # resumed decode step at that length, 5 timed calls after eight warm-up calls)
     sweep = {}
     if args.sweep and shape_name == "32b" and not args.layers:
         for length in (512, 2048, 8192, 16384):
@@ -493,6 +494,20 @@ def run_ours(args):
             sweep[str(length)] = {"ms_per_prefix": round(ms, 3), "tokens_per_s": round(length / (ms * 1e-3), 1),
                                   "tflops": round(fl / (ms * 1e-3) / 1e12, 1),
                                   "bar_ms_60pct_of_burst": round(fl / (0.6 * peaks()["bf16_tflops"] * 1e12) * 1e3, 1)}
+            # the resumed decode step at this length's resume position n = prefix + prefix / 8 (the suffix pages hold
+            # whatever finite K/V earlier runs left there: the step's cost does not depend on the values)
+            n_l = length + length // 8
+            table_d = perm_tgt[: n_l // bs + 1].copy()
+            ws_dl = model.workspace(kv.KV_OP_DECODE, n_l + 1)
+            for _ in range(8):      # long enough for the memory system to recover from the power-capped prefill
+                kv.kv_decode_step(model, tgt, int(ids_l[0]), n_l, table_d, logits, workspace=ws_dl)
+            torch.cuda.synchronize()
+            e0.record(stream)
+            for _ in range(5):
+                kv.kv_decode_step(model, tgt, int(ids_l[0]), n_l, table_d, logits, workspace=ws_dl)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            sweep[str(length)]["decode_step_ms_at_resume"] = round(e0.elapsed_time(e1) / 5, 3)
 
     if rank != 0:
         if world > 1:
