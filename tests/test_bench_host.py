@@ -61,3 +61,23 @@ def test_step_work_adds_up():
     assert w["pack"][0] == 2 * 32 * 64 * 2 * 32768 == w["unpack"][0]       # 128 MiB read + 128 MiB written
     assert w["decode_gemv"][0] / 1e9 == pytest.approx(62.41, abs=0.01)     # every layer's weights once
     assert w["rmsnorm"][0] == 127 * 4096 * 5120 * 6
+
+
+def test_documented_commands_name_existing_cases():
+    """Every `python profile_case.py <case>` and `bench.py --workload <name>` quoted in profiles/ and the documents
+    names a case or workload the scripts know (the commands must stay runnable as written)."""
+    import glob
+    import os
+    import re
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    texts = [open(f).read() for f in glob.glob(os.path.join(root, "profiles", "*.md"))]
+    texts += [open(os.path.join(root, f)).read() for f in ("DESIGN.md", "README.md", "BASELINE.md")]
+    text = "\n".join(texts)
+    source = open(os.path.join(root, "profile_case.py")).read()
+    cases = set(re.findall(r"python profile_case\.py ([a-z_]+)", text))
+    assert cases, "no profile command found"
+    for case in cases:
+        assert f'"{case}"' in source, case
+    bench_src = open(os.path.join(root, "bench.py")).read()
+    for name in set(re.findall(r"bench\.py --workload ([a-z0-9-]+)", text)):
+        assert name in bench.WORKLOADS or f'"{name}"' in bench_src, name
