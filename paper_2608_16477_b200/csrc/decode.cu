@@ -298,8 +298,8 @@ __global__ void __launch_bounds__(kPaSplitKeys, 2) paged_attention_split_kernel(
   // K and V rows of a tile into shared memory.  A warp copies its 32 rows (keys 32w..32w+31, the ones its MMAs
   // read) 32 / CH rows at a time: CH consecutive lanes cover one row's CH 16-byte chunks, so every instruction
   // moves whole rows (contiguous 2 D bytes each) instead of one chunk of 32 different rows.  Rows past the end
-  // repeat the last key (finite data, masked below).  Two commit groups: K first, then V.
-  auto load_tile = [&](int t) {
+  // repeat the last key (finite data, masked below).  One commit group per call (kv = 0: the K rows, 1: the V rows).
+  auto load_rows = [&](int t, int kv) {
     constexpr int RPI = 32 / CH;              // rows per instruction
     const int sub = lane / CH, c = lane % CH;
     const int bsz = cache.block_size;
@@ -307,24 +307,22 @@ __global__ void __launch_bounds__(kPaSplitKeys, 2) paged_attention_split_kernel(
     const int jk = min(t * kPaSplitKeys + warp * 32 + lane, n_ctx - 1);
     const int my_blk = block_table[jk / bsz];
     const int my_slot = jk % bsz;
+    const uint32_t tile = (uint32_t)__cvta_generic_to_shared(kv == 0 ? k_tile : v_tile);
 #pragma unroll
-    for (int kv = 0; kv < 2; ++kv) {
-      const uint32_t tile = (uint32_t)__cvta_generic_to_shared(kv == 0 ? k_tile : v_tile);
-#pragma unroll
-      for (int i = 0; i < CH; ++i) {
-        const int rw = i * RPI + sub;                        // row inside the warp's 32
-        const int r = warp * 32 + rw;                        // row of the tile
-        const int blk = __shfl_sync(0xffffffffu, my_blk, rw);
-        const int slot = __shfl_sync(0xffffffffu, my_slot, rw);
-        const bf16 *src = reinterpret_cast<const bf16 *>(cache.page(layer, kv, blk)) +
-                          ((long long)slot * cache.n_kv_heads + g) * D + c * 8;
-        const uint32_t pc = (uint32_t)((c & ~7) | ((c ^ r) & 7)) * 16;
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(tile + r * RB + pc), "l"(src) : "memory");
-      }
-      asm volatile("cp.async.commit_group;" ::: "memory");
+    for (int i = 0; i < CH; ++i) {
+      const int rw = i * RPI + sub;                        // row inside the warp's 32
+      const int r = warp * 32 + rw;                        // row of the tile
+      const int blk = __shfl_sync(0xffffffffu, my_blk, rw);
+      const int slot = __shfl_sync(0xffffffffu, my_slot, rw);
+      const bf16 *src = reinterpret_cast<const bf16 *>(cache.page(layer, kv, blk)) +
+                        ((long long)slot * cache.n_kv_heads + g) * D + c * 8;
+      const uint32_t pc = (uint32_t)((c & ~7) | ((c ^ r) & 7)) * 16;
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(tile + r * RB + pc), "l"(src) : "memory");
     }
+    asm volatile("cp.async.commit_group;" ::: "memory");
   };
-  load_tile(t_begin);
+  load_rows(t_begin, 0);
+  load_rows(t_begin, 1);
   const uint32_t k_s = (uint32_t)__cvta_generic_to_shared(k_tile);
   const uint32_t v_s = (uint32_t)__cvta_generic_to_shared(v_tile);
   const int r0 = lane >> 2, cq = (lane & 3) * 2;       // fragment row (and row + 8), first of two columns
@@ -361,6 +359,9 @@ __global__ void __launch_bounds__(kPaSplitKeys, 2) paged_attention_split_kernel(
 
     for (int t = t_begin; t < t_end; ++t) {
       const int n_keys = min(n_ctx - t * kPaSplitKeys, kPaSplitKeys);
+      // the tile that follows: the next one of this pass, or the first one again for the next pass of heads (a single
+      // tile stays where it is)
+      const int t_next = one_tile ? -1 : (t + 1 < t_end ? t + 1 : (h0 + kPaRows < group ? t_begin : -1));
       asm volatile("cp.async.wait_group 1;" ::: "memory");      // K rows have landed
       __syncthreads();      // (also: the previous tile or pass no longer reads the row statistics and o_red)
       // ---- S = Q K^T for this warp's 32 keys: 4 n-tiles of 8 keys
@@ -401,6 +402,7 @@ __global__ void __launch_bounds__(kPaSplitKeys, 2) paged_attention_split_kernel(
       }
       asm volatile("cp.async.wait_group 0;" ::: "memory");      // V rows have landed
       __syncthreads();
+      if (t_next >= 0) load_rows(t_next, 0);      // every warp is done with this tile's K: the next K rows travel under P V
       mx0 = run0;
       mx1 = run1;
 #pragma unroll
@@ -449,10 +451,9 @@ __global__ void __launch_bounds__(kPaSplitKeys, 2) paged_attention_split_kernel(
           mma_bf16_16816(oc[nt + 1], pl[kk], bfr[2], bfr[3]);
         }
       }
-      // the next tile of this pass, or the first tile again for the next pass of heads (a single tile stays where it is)
-      if (!one_tile && (t + 1 < t_end || h0 + kPaRows < group)) {
-        __syncthreads();      // every warp is done with this tile's K and V
-        load_tile(t + 1 < t_end ? t + 1 : t_begin);
+      if (t_next >= 0) {
+        __syncthreads();      // every warp is done with this tile's V
+        load_rows(t_next, 1);
       }
     }
     // ---- the four warps' shares of O and of the row sums meet in shared memory
